@@ -1,0 +1,352 @@
+"""Pins for the CPU oracle: each test fixes the oracle to something other than itself
+(hand arithmetic, brute force, a lemma, a closed form, the paper's printed table)."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import routerelay_oracle as O
+from paper_2609_07306_b200 import workload as W
+
+
+def _params(w, **kw):
+    base = dict(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, gamma=w.gamma, causal=w.causal,
+                causal_offset=0, seed=w.seed)
+    base.update(kw)
+    return O.OracleParams(**base)
+
+
+def _load_rows(path):
+    rows = []
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+# ------------------------------------------------------------------ Eq. 1
+def test_scores_hand_computed():
+    # Eq. 1 on a 2x3 problem with d=2, worked by hand:
+    q = np.array([[1.0, 2.0], [-1.0, 0.5]])
+    k = np.array([[3.0, 4.0], [0.0, -1.0], [2.0, 2.0]])
+    p = O.OracleParams(n_q=2, n_k=3, k=1, m=1, r=0)
+    s = O.scores(q, k, p)
+    expect = np.array([[11.0, -2.0, 6.0], [-1.0, -0.5, -1.0]])
+    assert np.array_equal(s, expect)
+    # transposed operands or a 1/sqrt(d) factor would give different numbers
+    assert s[0, 0] == 1 * 3 + 2 * 4
+
+
+def test_scores_causal_mask_and_offset():
+    q = np.ones((4, 2))
+    k = np.ones((4, 2))
+    s = O.scores(q, k, O.OracleParams(n_q=4, n_k=4, k=1, m=0, r=0, causal=True))
+    for i in range(4):
+        assert np.all(s[i, : i + 1] == 2.0) and np.all(np.isneginf(s[i, i + 1:]))
+    s = O.scores(q[:2], k, O.OracleParams(n_q=2, n_k=4, k=1, m=0, r=0, causal=True,
+                                           causal_offset=2))
+    assert np.isfinite(s[0]).sum() == 3 and np.isfinite(s[1]).sum() == 4
+
+
+# ------------------------------------------------------------------ Eq. 2 + Sec 3.1 near-miss
+def _brute_rank(s_row, v):
+    return [j for _, j in sorted((-float(s_row[j]), j) for j in range(v))]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_topk_nearmiss_bruteforce(seed):
+    rng = np.random.default_rng(seed)
+    n_k = int(rng.integers(3, 17))
+    # coarse values force many exact ties
+    s_row = rng.integers(-3, 4, size=n_k).astype(np.float64) / 4.0
+    for v in range(1, n_k + 1):
+        brute = _brute_rank(s_row, v)
+        assert list(O.rank_order(s_row, v)) == brute
+        for k in range(1, n_k + 1):
+            for m in (0, 1, 3):
+                p = O.OracleParams(n_q=1, n_k=n_k, k=k, m=m, r=0)
+                route, sent, kth, margin = O.route_row(s_row, v, p, g=0, layer=0)
+                kk = min(k, v)
+                assert [j for j in route if j >= 0] == brute[:kk]
+                assert [j for j in sent if j >= 0] == brute[kk:kk + m]
+                assert kth == s_row[brute[kk - 1]]
+                if v > kk:
+                    assert margin == s_row[brute[kk - 1]] - s_row[brute[kk]]
+                    # Sec 3.3: min selected - max unselected
+                    assert margin == min(s_row[j] for j in brute[:kk]) - \
+                        max(s_row[j] for j in brute[kk:v])
+                else:
+                    assert margin == float("inf")
+
+
+def test_topk_matches_library_when_no_ties():
+    rng = np.random.default_rng(7)
+    s = rng.standard_normal((32, 200))
+    for i in range(32):
+        lib = set(np.argpartition(-s[i], 12)[:12].tolist())
+        assert set(O.full_route(s[i], 200, 12).tolist()) == lib
+
+
+def test_negative_zero_ties_with_positive_zero():
+    q = np.array([[0.0, 1.0]])
+    k = np.array([[-1.0, 0.0], [1.0, 0.0], [0.0, -1.0]])     # scores: -0.0, +0.0, -1
+    p = O.OracleParams(n_q=1, n_k=3, k=1, m=1, r=0)
+    s = O.scores(q, k, p)
+    assert list(O.rank_order(s[0], 3)) == [0, 1, 2]           # tie -> smaller index first
+
+
+# ------------------------------------------------------------------ Lemma 1
+@pytest.mark.parametrize("seed", range(5))
+def test_lemma1_margin_stability(seed):
+    rng = np.random.default_rng(100 + seed)
+    n_k, k, m, r = 96, 8, 4, 4
+    p = O.OracleParams(n_q=1, n_k=n_k, k=k, m=m, r=r, seed=seed)
+    s_row = rng.standard_normal(n_k)
+    route, sent, kth, margin = O.route_row(s_row, n_k, p, g=3, layer=0)
+    assert margin > 0
+    # any perturbation with sup-norm < margin/2 keeps the route and does not trigger
+    for _ in range(20):
+        e = rng.uniform(-1, 1, n_k)
+        e *= 0.49 * margin / np.abs(e).max()
+        s2 = s_row + e
+        assert set(O.full_route(s2, n_k, k)) == set(route)
+        led = O.Ledger.empty(1, p)
+        led.routes[0], led.sentinels[0], led.ages[0] = route, sent, 0
+        _, a, b, _ = O.candidate_scores(s2[None, :], led.routes, led.sentinels)
+        assert a[0] > b[0]
+    # adversarial perturbation just above margin/2 on the k-th / (k+1)-th pair flips the set
+    order = O.rank_order(s_row, n_k)
+    e = np.zeros(n_k)
+    e[order[k - 1]] = -0.51 * margin
+    e[order[k]] = +0.51 * margin
+    s3 = s_row + e
+    assert set(O.full_route(s3, n_k, k)) != set(route)
+    _, a, b, _ = O.candidate_scores(s3[None, :], route[None, :], sent[None, :])
+    assert not (a[0] > b[0])          # and the near-miss sentinel catches it
+
+
+def test_lemma1_query_level_perturbation():
+    rng = np.random.default_rng(5)
+    d, n_k, k = 16, 64, 6
+    kk = rng.standard_normal((n_k, d))
+    q = rng.standard_normal((1, d))
+    p = O.OracleParams(n_q=1, n_k=n_k, k=k, m=3, r=0)
+    s = O.scores(q, kk, p)
+    route, _, _, margin = O.route_row(s[0], n_k, p, 0, 0)
+    dq = rng.standard_normal((1, d))
+    # |dq . k_j| <= ||dq|| max||k_j|| = eps < margin/2
+    dq *= 0.49 * margin / (np.linalg.norm(dq) * np.linalg.norm(kk, axis=1).max())
+    s2 = O.scores(q + dq, kk, p)
+    assert np.abs(s2 - s).max() <= 0.5 * margin
+    assert set(O.full_route(s2[0], n_k, k)) == set(route)
+
+
+# ------------------------------------------------------------------ trigger invariants
+def _run(w, problems, **over):
+    q, k = W.generate(w, problems=problems)
+    p = _params(w, **over)
+    res, summ = O.run_layers(W.as_float32(q), W.as_float32(k), p, w.anchor_every,
+                             problem_ids=problems, keep_scores=True)
+    return p, res, summ
+
+
+@pytest.mark.parametrize("wl,problems", [(W.tiny(), [0]), (W.moderate(), [0, 5])])
+def test_trigger_invariants(wl, problems):
+    p, res, summ = _run(wl, problems)
+    v = np.tile(p.valid_counts(), len(problems))
+    lost_on_flagged = 0
+    for l in range(1, len(res)):
+        cur, prev = res[l], res[l - 1]
+        if cur.is_anchor:
+            assert np.all(cur.flags == 1) and np.all(cur.ledger.ages == 0)
+            assert len(cur.refresh_rows) == len(v)
+            continue
+        stable = cur.flags == 0
+        # (i) unflagged: route and sentinels relayed bit-identically, age advances
+        assert np.array_equal(cur.ledger.routes[stable], prev.ledger.routes[stable])
+        assert np.array_equal(cur.ledger.sentinels[stable], prev.ledger.sentinels[stable])
+        assert np.array_equal(cur.ledger.ages[stable], prev.ledger.ages[stable] + 1)
+        # (ii) flagged: route = exact TopK of this layer, age 0
+        fl = ~stable
+        assert np.array_equal(cur.ledger.routes[fl], cur.full_routes[fl])
+        assert np.all(cur.ledger.ages[fl] == 0)
+        # compaction order: ascending ids of the flagged rows, nothing else
+        assert np.array_equal(cur.refresh_rows, np.nonzero(cur.flags)[0])
+        # (iii) gamma = 0: a flagged row's exact TopK differs from the stale route unless an
+        # exact tie sits on the boundary (no false positives of the trigger)
+        for gr in np.nonzero(fl)[0]:
+            if cur.alpha[gr] == cur.beta[gr]:
+                continue
+            old = set(int(j) for j in prev.ledger.routes[gr] if j >= 0)
+            new = set(int(j) for j in cur.full_routes[gr] if j >= 0)
+            assert old != new
+        # rows that can select everything they see carry no sentinels and never flag
+        assert not np.any(cur.flags[v <= p.k])
+        # (iv) recall is lost on unflagged rows only
+        h, t = O.recall_counts(cur.ledger.routes[fl], cur.full_routes[fl])
+        lost_on_flagged += t - h
+    assert lost_on_flagged == 0
+    assert 0.0 < summ.flagged_relay_fraction < 1.0
+    assert summ.recall_all >= summ.recall_relay * (1 - 1e-12) or summ.recall_relay == 1.0
+
+
+def test_no_sentinels_is_fixed_stride_reuse():
+    # m = r = 0: nothing can challenge -> pure reuse between anchors ("fixed stride")
+    w = W.tiny().replace(m=0, r=0)
+    p, res, summ = _run(w, [0])
+    assert summ.flagged_relay_fraction == 0.0
+    for l in range(1, len(res)):
+        assert np.array_equal(res[l].ledger.routes, res[0].ledger.routes)
+        assert np.all(res[l].ledger.ages == l)
+
+
+def test_infinite_guard_margin_is_route_every_layer():
+    w = W.tiny()
+    p, res, summ = _run(w, [0], gamma=float("inf"))
+    assert summ.recall_all == 1.0
+    for l in range(1, len(res)):
+        assert np.all(res[l].flags == 1)
+        assert np.array_equal(res[l].ledger.routes, res[l].full_routes)
+
+
+def test_zero_drift_never_flags():
+    w = W.tiny().replace(rho=0.0)
+    p, res, summ = _run(w, [0])
+    assert summ.flagged_relay_fraction == 0.0 and summ.recall_all == 1.0
+    for l in range(1, len(res)):
+        assert np.array_equal(res[l].ledger.routes, res[0].ledger.routes)
+
+
+def test_flagged_fraction_grows_with_drift():
+    fr = []
+    for rho in (0.01, 0.05, 0.2):
+        _, _, summ = _run(W.tiny().replace(rho=rho), [0])
+        fr.append(summ.flagged_relay_fraction)
+    assert fr[0] <= fr[1] <= fr[2] and fr[0] < fr[2]
+
+
+# ------------------------------------------------------------------ random sentinels
+def test_finaliser_published_vectors(golden_dir):
+    vec = [int(r[0]) for r in _load_rows(os.path.join(golden_dir, "splitmix64_vectors.txt"))]
+    state = 1234567
+    for expect in vec:
+        state = (state + 0x9E3779B97F4A7C15) & ((1 << 64) - 1)
+        assert O.fmix64(state) == expect
+
+
+def test_sampler_invariants_and_small_pools():
+    for v in range(1, 40):
+        for n_ex in range(0, min(v, 20) + 1):
+            excluded = list(range(0, 2 * n_ex, 2))[:n_ex]
+            excluded = [j for j in excluded if j < v]
+            pool = [j for j in range(v) if j not in excluded]
+            for r in (0, 1, 4, 9):
+                out = O.draw_random_sentinels(excluded, v, r, seed=3, g=v * 131 + n_ex, layer=2)
+                assert len(out) == min(r, len(pool))
+                assert len(set(out)) == len(out)
+                assert all(0 <= j < v and j not in excluded for j in out)
+                if len(pool) <= r:
+                    assert out == pool          # whole pool, ascending, no RNG involved
+
+
+def test_sampler_depends_on_seed_row_layer():
+    ex = list(range(12))
+    a = O.draw_random_sentinels(ex, 512, 8, 1, 10, 3)
+    assert a != O.draw_random_sentinels(ex, 512, 8, 2, 10, 3)
+    assert a != O.draw_random_sentinels(ex, 512, 8, 1, 11, 3)
+    assert a != O.draw_random_sentinels(ex, 512, 8, 1, 10, 4)
+    assert a == O.draw_random_sentinels(ex, 512, 8, 1, 10, 3)
+
+
+def test_sampler_uniform_and_miss_probability():
+    """Eq. 6: P(miss) = C(N-u, r) / C(N, r) for r draws without replacement from a pool of N
+    that hides u challengers; plus chi-square uniformity over the pool."""
+    from scipy import stats
+    v, r, u = 64, 8, 5
+    excluded = list(range(0, 32, 2))                 # 16 excluded -> N = 48
+    pool = [j for j in range(v) if j not in excluded]
+    N = len(pool)
+    challengers = set(pool[3::10][:u])
+    assert len(challengers) == u
+    rows = 30000
+    counts = dict.fromkeys(pool, 0)
+    miss = 0
+    for g in range(rows):
+        out = O.draw_random_sentinels(excluded, v, r, seed=11, g=g, layer=1)
+        for j in out:
+            counts[j] += 1
+        miss += not challengers.intersection(out)
+    p_exact = math.comb(N - u, r) / math.comb(N, r)
+    assert p_exact <= (1 - u / N) ** r                # the paper's upper bound
+    sigma = math.sqrt(p_exact * (1 - p_exact) / rows)
+    assert abs(miss / rows - p_exact) < 4 * sigma
+    chi2 = stats.chisquare(list(counts.values()))
+    assert chi2.pvalue > 1e-4
+    # a sampler that drew WITH replacement would have a visibly different miss rate
+    assert abs((1 - u / N) ** r - p_exact) > 8 * sigma
+
+
+# ------------------------------------------------------------------ work accounting
+def test_score_pair_definition_matches_paper_table(golden_dir):
+    """The paper's sentinel-ablation table fixes what 'score pairs' and 'rerouted rows'
+    count: given its rerouted-row column, the accounting must reproduce its score-pair
+    column (values printed to 0.1 %)."""
+    L, n, k = 24, 256, 12
+    for m, r, rer_pct, pairs_pct in _load_rows(os.path.join(golden_dir,
+                                                            "sentinel_ablation_table.txt")):
+        m, r, rer_pct, pairs_pct = int(m), int(r), float(rer_pct), float(pairs_pct)
+        p = O.OracleParams(n_q=n, n_k=n, k=k, m=m, r=r)
+        flagged_total = int(round(rer_pct / 100 * L * n - n))
+        kinds = [True] + [False] * (L - 1)
+        flags = [np.ones(n, np.uint8)]
+        left = flagged_total
+        for l in range(1, L):
+            f = np.zeros(n, np.uint8)
+            take = min(n, -(-left // (L - l)))
+            f[:take] = 1
+            left -= take
+            flags.append(f)
+        cc = [None] + [np.full(n, p.c)] * (L - 1)
+        c = O.work_counters(p, 1, kinds, flags, cc)
+        rerouted, flagged, pairs = O.fractions_from_counters(c)
+        assert abs(100 * rerouted - rer_pct) < 0.06
+        assert abs(100 * pairs - pairs_pct) < 0.06, (m, r, 100 * pairs)
+
+
+def test_ledger_size(golden_dir):
+    (n_q, c, nbytes), = _load_rows(os.path.join(golden_dir, "ledger_size.txt"))
+    p = O.OracleParams(n_q=int(n_q), n_k=4096, k=32, m=16, r=16)
+    assert p.c == int(c)
+    assert O.Ledger.empty(int(n_q), p).index_bytes() == int(nbytes)
+
+
+def test_counters_consistent_with_run():
+    w = W.moderate()
+    p, res, summ = _run(w, [1])
+    c = summ.counters
+    v = p.valid_counts()
+    n_anchor = sum(r.is_anchor for r in res)
+    assert c["anchor_rows"] == n_anchor * w.n_q
+    assert c["dense_pairs"] == len(res) * int(v.sum())
+    assert c["flagged_rows"] == sum(int(r.flags.sum()) for r in res if not r.is_anchor)
+    # causal rows with v_i <= k have v_i candidates, later rows up to c
+    first_relay = res[1]
+    assert first_relay.cand_scores.shape == (w.n_q, w.c)
+    assert np.isfinite(first_relay.cand_scores[0]).sum() == 1
+    assert np.isfinite(first_relay.cand_scores[-1]).sum() == w.c
+
+
+def test_token_ranges():
+    routes = np.array([[5, 2, -1], [0, 7, 3]], np.int32)
+    tr = O.token_ranges(routes, 64)
+    assert tr[0].tolist() == [[128, 192], [320, 384], [-1, -1]]
+    assert tr[1].tolist() == [[0, 64], [192, 256], [448, 512]]
+
+
+def test_relay_requires_anchor():
+    p = O.OracleParams(n_q=4, n_k=4, k=1, m=1, r=0)
+    with pytest.raises(ValueError):
+        O.relay_layer(O.Ledger.empty(4, p), np.ones((1, 4, 2)), np.ones((1, 4, 2)), p, 1)
