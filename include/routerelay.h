@@ -1,0 +1,169 @@
+/*
+ * routerelay.h -- C ABI of the B200 (sm_100a) route-maintenance library.
+ *
+ * The library maintains, on the device, the RouteRelay "route ledger" of a batch of
+ * independent routing problems (one per batch x head pair) across Transformer layers:
+ *
+ *   anchor layer : full chunk routing  S = Qc Kc^T (Eq. 1), per-row TopK (Eq. 2), and a
+ *                  ledger of each row's k selected chunks, its m near-miss chunks and r
+ *                  seeded random sentinels (Section 3.1);
+ *   relay layer  : rescoring of route + sentinels against the current layer's Qc/Kc
+ *                  (Section 3.2), the challenge test alpha > beta + gamma (Eq. 5),
+ *                  prefix-sum compaction of the failing rows, full re-routing of exactly
+ *                  those rows, and the ledger update (Sections 4.1, 4.2).
+ *
+ * Conventions
+ *   - Every function returns an int status: RR_OK (0) or a negative RR_ERR_* code.  Nothing
+ *     throws, aborts or traps.  rr_strerror() names a code.
+ *   - "device pointer" means memory of the CUDA device that was current when
+ *     rr_ledger_init() ran; "host pointer" means ordinary (preferably pinned) host memory.
+ *   - The library allocates no device memory.  The caller owns the ledger buffer and the
+ *     scratch buffer (sizes from rr_workspace_bytes) and must keep them alive, and must not
+ *     touch them while work is in flight, until rr_ledger_destroy().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     rr_route_anchor / rr_route_relay only enqueue work: they never synchronise with the
+ *     host.  Results are read through rr_ledger_views() after the caller has synchronised
+ *     the stream.
+ *   - Qc is [batch, heads, n_q, d], Kc is [batch, heads, n_k, d], contiguous row-major,
+ *     16-byte aligned, dtype per rr_config.dtype; both are borrowed until the enqueued work
+ *     has finished.
+ *   - Row ids are global: g = problem * n_q + i with problem = batch_index * heads + head.
+ *   - Chunk ids are int32; a slot a row cannot fill (fewer valid chunks than k, m or r)
+ *     holds -1.  The order of ids inside a route / near-miss / random group carries no
+ *     meaning (the paper defines them as sets).
+ *   - Ties in TopK break towards the smaller chunk id; -0.0 equals +0.0.
+ */
+#ifndef ROUTERELAY_H_
+#define ROUTERELAY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RR_OK                 0
+#define RR_ERR_INVALID_ARG   -1   /* null pointer, negative size, misaligned buffer, ...        */
+#define RR_ERR_UNSUPPORTED   -2   /* shape / dtype outside what the kernels are built for      */
+#define RR_ERR_STATE         -3   /* e.g. relay on a ledger that was never anchored            */
+#define RR_ERR_CUDA          -4   /* a CUDA runtime call failed (see rr_last_cuda_error)       */
+#define RR_ERR_TIMEOUT       -5   /* a bounded device-side wait expired (device status word)   */
+#define RR_ERR_TOO_SMALL     -6   /* caller-provided buffer smaller than required              */
+
+#define RR_BF16 0
+#define RR_F32  1
+
+/* bits of the device status word (rr_ledger_status) */
+#define RR_STATUS_TIMEOUT      1u  /* an mbarrier wait in a kernel gave up                     */
+#define RR_STATUS_BAD_INDEX    2u  /* a ledger entry outside [0, v_i) was met and skipped      */
+#define RR_STATUS_OVERFLOW     4u  /* an internal per-row buffer overflowed (result invalid)   */
+
+typedef struct rr_ledger rr_ledger;   /* opaque; owns only a small host struct */
+
+/* One routing configuration.  P = batch*heads independent problems, rows = P*n_q. */
+typedef struct rr_config {
+  int32_t batch, heads;
+  int32_t n_q, n_k;        /* query chunks / key chunks per problem                        */
+  int32_t d;               /* representation width: 64 or 128                              */
+  int32_t k, m, r;         /* route width (Eq. 2), near-miss and random sentinels (Sec 3.1)*/
+  int32_t dtype;           /* RR_BF16 or RR_F32 (inputs; accumulation is always fp32)      */
+  int32_t causal;          /* 0: every row sees all n_k chunks; 1: row i sees chunks
+                              j < min(n_k, i + 1 + causal_offset)                          */
+  int32_t causal_offset;
+  float   gamma;           /* guard margin of Eq. 5, >= 0 (+inf allowed)                   */
+  uint64_t seed;           /* seed of the random-sentinel sampler                          */
+  int32_t chunk_tokens;    /* >0: also expand routes to token ranges of this chunk size    */
+  int32_t debug_outputs;   /* 1: relay also stores every candidate score (tests)           */
+} rr_config;
+
+/* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */
+typedef struct rr_views {
+  int32_t* routes;          /* [rows, k]     selected chunk ids                             */
+  int32_t* sentinels;       /* [rows, m+r]   near-miss (first m) then random (last r)       */
+  int32_t* ages;            /* [rows]        layers since the row was last fully routed; -1 after reset */
+  float*   kth_score;       /* [rows]        weakest selected score when last routed        */
+  float*   margin;          /* [rows]        Section 3.3 margin when last routed (+inf if nothing is unselected) */
+  uint8_t* flags;           /* [rows]        1 = row failed Eq. 5 at the last relay (anchor: all 1) */
+  float*   alpha;           /* [rows]        min route score at the last relay              */
+  float*   beta;            /* [rows]        max sentinel score at the last relay (-inf if none) */
+  int32_t* refresh_rows;    /* [rows]        ascending global ids of the flagged rows       */
+  int32_t* refresh_count;   /* [1]           how many (= rho_l * rows)                      */
+  int32_t* problem_offsets; /* [P+1]         exclusive scan of per-problem flagged counts   */
+  int32_t* token_ranges;    /* [rows, k, 2]  [start,end) per route slot, ascending chunk id; NULL if chunk_tokens==0 */
+  float*   cand_scores;     /* [rows, k+m+r] candidate scores of the last relay; NULL unless debug_outputs */
+  uint64_t* counters;       /* [RR_NUM_COUNTERS] cumulative since reset, see below          */
+  uint32_t* status;         /* [1]           RR_STATUS_* bits                               */
+} rr_views;
+
+/* counters[] indices: work accounting in the sense of the paper's "rerouted rows" and
+ * "score pairs" columns (Section 5): anchors charge every row its full row; relays charge
+ * every row its candidates and every flagged row its full row in addition. */
+#define RR_CNT_LAYER_CALLS   0
+#define RR_CNT_ANCHOR_ROWS   1
+#define RR_CNT_RELAY_ROWS    2
+#define RR_CNT_FLAGGED_ROWS  3
+#define RR_CNT_CAND_PAIRS    4
+#define RR_CNT_FULL_PAIRS    5
+#define RR_CNT_DENSE_PAIRS   6   /* what full routing on every layer would have scored        */
+#define RR_NUM_COUNTERS      8
+
+/* Sizes of the two caller-owned device buffers for a configuration.  Host-only. */
+int rr_workspace_bytes(const rr_config* cfg, size_t* ledger_bytes, size_t* scratch_bytes);
+
+/* Creates the host handle over caller-owned device buffers (both 256-byte aligned, at least
+ * the sizes rr_workspace_bytes reports).  Does not touch the buffers: call rr_ledger_reset. */
+int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
+                   void* dev_scratch, size_t scratch_bytes, rr_ledger** out);
+
+/* Enqueues: routes/sentinels = -1, ages = -1, counters = 0, status = 0. */
+int rr_ledger_reset(rr_ledger* L, void* stream);
+
+/* Frees the host handle only. */
+int rr_ledger_destroy(rr_ledger* L);
+
+/* Anchor layer (Section 4.1: "constructs this state from a complete chunk-score matrix").
+ * Routes every row, rebuilds all sentinels with the sampler keyed by (seed, row, layer),
+ * sets ages to 0, flags to 1, refresh_rows to all rows.  qc, kc: device pointers. */
+int rr_route_anchor(rr_ledger* L, const void* qc, const void* kc, int32_t layer, void* stream);
+
+/* Relay layer (Sections 3.2, 4.1, 4.2).  Requires a previous anchor (else RR_ERR_STATE).
+ * The flagged-row list, its count and the refresh all stay on the device. */
+int rr_route_relay(rr_ledger* L, const void* qc, const void* kc, int32_t layer, void* stream);
+
+/* One layer driven from HOST buffers: copies qc/kc (host pointers, same layout) into the
+ * caller's device staging buffers, runs the anchor (is_anchor != 0) or relay step, and
+ * copies the routes [rows,k] back to host_routes (may be NULL).  All on `stream`, no host
+ * synchronisation inside; the caller synchronises before reading host_routes. */
+int rr_route_layer_host(rr_ledger* L, const void* host_qc, const void* host_kc,
+                        void* dev_qc_staging, void* dev_kc_staging, int32_t layer,
+                        int32_t is_anchor, int32_t* host_routes, void* stream);
+
+/* Device pointers to state and per-layer outputs. */
+int rr_ledger_views(rr_ledger* L, rr_views* out);
+
+/* Checkpoint / restore of the ledger (routes, sentinels, ages, kth_score, margin) to a host
+ * blob of rr_export_bytes() bytes, laid out in that order, each array as in rr_views.
+ * Both synchronise `stream`. */
+int rr_export_bytes(const rr_config* cfg, size_t* bytes);
+int rr_ledger_export(rr_ledger* L, void* host_blob, size_t bytes, void* stream);
+int rr_ledger_import(rr_ledger* L, const void* host_blob, size_t bytes, void* stream);
+
+/* Synchronous read of the device status word (RR_STATUS_* bits); RR_ERR_TIMEOUT is
+ * returned if the timeout bit is set. */
+int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out);
+
+/* Host-callable copy of the sampler's counter-based generator (the t-th 32-bit draw of
+ * global row g when its sentinels are rebuilt at `layer`); same code the kernels run. */
+uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t t);
+
+/* How many kernels the library has launched since it was loaded (all ledgers). */
+uint64_t rr_kernel_launch_count(void);
+
+const char* rr_strerror(int code);
+const char* rr_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROUTERELAY_H_ */

@@ -1,0 +1,180 @@
+"""ctypes binding of librouterelay.so -- argument marshalling only.
+
+Every function here has the name of the C entry point it wraps (include/routerelay.h).
+Nothing is computed in Python, and there is no fallback: if the shared library is missing
+or fails to load, importing the symbols raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "librouterelay.so")
+
+RR_OK = 0
+RR_ERR_INVALID_ARG = -1
+RR_ERR_UNSUPPORTED = -2
+RR_ERR_STATE = -3
+RR_ERR_CUDA = -4
+RR_ERR_TIMEOUT = -5
+RR_ERR_TOO_SMALL = -6
+RR_BF16 = 0
+RR_F32 = 1
+RR_STATUS_TIMEOUT = 1
+RR_STATUS_BAD_INDEX = 2
+RR_STATUS_OVERFLOW = 4
+RR_NUM_COUNTERS = 8
+COUNTER_NAMES = ("layer_calls", "anchor_rows", "relay_rows", "flagged_rows", "cand_pairs",
+                 "full_pairs", "dense_pairs")
+
+
+class rr_config(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("heads", C.c_int32), ("n_q", C.c_int32),
+                ("n_k", C.c_int32), ("d", C.c_int32), ("k", C.c_int32), ("m", C.c_int32),
+                ("r", C.c_int32), ("dtype", C.c_int32), ("causal", C.c_int32),
+                ("causal_offset", C.c_int32), ("gamma", C.c_float), ("seed", C.c_uint64),
+                ("chunk_tokens", C.c_int32), ("debug_outputs", C.c_int32)]
+
+
+class rr_views(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "routes", "sentinels", "ages", "kth_score", "margin", "flags", "alpha", "beta",
+        "refresh_rows", "refresh_count", "problem_offsets", "token_ranges", "cand_scores",
+        "counters", "status")]
+
+
+class RouteRelayError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = f"{where}: {strerror(code)} ({code})"
+        if code == RR_ERR_CUDA:
+            msg += ": " + last_cuda_error()
+        super().__init__(msg)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_07306_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+        cfgp = C.POINTER(rr_config)
+        L.rr_workspace_bytes.argtypes = [cfgp, C.POINTER(sz), C.POINTER(sz)]
+        L.rr_export_bytes.argtypes = [cfgp, C.POINTER(sz)]
+        L.rr_ledger_init.argtypes = [cfgp, vp, sz, vp, sz, C.POINTER(vp)]
+        L.rr_ledger_reset.argtypes = [vp, vp]
+        L.rr_ledger_destroy.argtypes = [vp]
+        L.rr_route_anchor.argtypes = [vp, vp, vp, i32, vp]
+        L.rr_route_relay.argtypes = [vp, vp, vp, i32, vp]
+        L.rr_route_layer_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.rr_ledger_views.argtypes = [vp, C.POINTER(rr_views)]
+        L.rr_ledger_export.argtypes = [vp, vp, sz, vp]
+        L.rr_ledger_import.argtypes = [vp, vp, sz, vp]
+        L.rr_ledger_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+        L.rr_sampler_draw_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
+        L.rr_sampler_draw_u32.restype = C.c_uint32
+        L.rr_kernel_launch_count.argtypes = []
+        L.rr_kernel_launch_count.restype = C.c_uint64
+        L.rr_strerror.argtypes = [C.c_int]
+        L.rr_strerror.restype = C.c_char_p
+        L.rr_last_cuda_error.argtypes = []
+        L.rr_last_cuda_error.restype = C.c_char_p
+        for name in ("rr_workspace_bytes", "rr_export_bytes", "rr_ledger_init", "rr_ledger_reset",
+                     "rr_ledger_destroy", "rr_route_anchor", "rr_route_relay",
+                     "rr_route_layer_host", "rr_ledger_views", "rr_ledger_export",
+                     "rr_ledger_import", "rr_ledger_status"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != RR_OK:
+        raise RouteRelayError(code, where)
+
+
+def strerror(code: int) -> str:
+    return lib().rr_strerror(code).decode()
+
+
+def last_cuda_error() -> str:
+    return lib().rr_last_cuda_error().decode()
+
+
+def rr_workspace_bytes(cfg: rr_config):
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(lib().rr_workspace_bytes(C.byref(cfg), C.byref(a), C.byref(b)), "rr_workspace_bytes")
+    return a.value, b.value
+
+
+def rr_export_bytes(cfg: rr_config) -> int:
+    a = C.c_size_t()
+    _check(lib().rr_export_bytes(C.byref(cfg), C.byref(a)), "rr_export_bytes")
+    return a.value
+
+
+def rr_ledger_init(cfg: rr_config, dev_ledger: int, ledger_bytes: int, dev_scratch: int,
+                   scratch_bytes: int) -> int:
+    h = C.c_void_p()
+    _check(lib().rr_ledger_init(C.byref(cfg), dev_ledger, ledger_bytes, dev_scratch,
+                                scratch_bytes, C.byref(h)), "rr_ledger_init")
+    return h.value
+
+
+def rr_ledger_reset(h: int, stream: int) -> None:
+    _check(lib().rr_ledger_reset(h, stream), "rr_ledger_reset")
+
+
+def rr_ledger_destroy(h: int) -> None:
+    _check(lib().rr_ledger_destroy(h), "rr_ledger_destroy")
+
+
+def rr_route_anchor(h: int, qc: int, kc: int, layer: int, stream: int) -> None:
+    _check(lib().rr_route_anchor(h, qc, kc, layer, stream), "rr_route_anchor")
+
+
+def rr_route_relay(h: int, qc: int, kc: int, layer: int, stream: int) -> None:
+    _check(lib().rr_route_relay(h, qc, kc, layer, stream), "rr_route_relay")
+
+
+def rr_route_layer_host(h: int, host_qc: int, host_kc: int, dev_qc: int, dev_kc: int,
+                        layer: int, is_anchor: bool, host_routes: int, stream: int) -> None:
+    _check(lib().rr_route_layer_host(h, host_qc, host_kc, dev_qc, dev_kc, layer,
+                                     1 if is_anchor else 0, host_routes, stream),
+           "rr_route_layer_host")
+
+
+def rr_ledger_views(h: int) -> rr_views:
+    v = rr_views()
+    _check(lib().rr_ledger_views(h, C.byref(v)), "rr_ledger_views")
+    return v
+
+
+def rr_ledger_export(h: int, host_blob: int, nbytes: int, stream: int) -> None:
+    _check(lib().rr_ledger_export(h, host_blob, nbytes, stream), "rr_ledger_export")
+
+
+def rr_ledger_import(h: int, host_blob: int, nbytes: int, stream: int) -> None:
+    _check(lib().rr_ledger_import(h, host_blob, nbytes, stream), "rr_ledger_import")
+
+
+def rr_ledger_status(h: int, stream: int) -> int:
+    s = C.c_uint32()
+    _check(lib().rr_ledger_status(h, stream, C.byref(s)), "rr_ledger_status")
+    return s.value
+
+
+def rr_sampler_draw_u32(seed: int, g: int, layer: int, t: int) -> int:
+    return int(lib().rr_sampler_draw_u32(seed, g, layer, t))
+
+
+def rr_kernel_launch_count() -> int:
+    return int(lib().rr_kernel_launch_count())

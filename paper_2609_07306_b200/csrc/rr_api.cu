@@ -1,0 +1,309 @@
+// C ABI of the route-maintenance library: handle management, buffer layout, and the two
+// layer calls (anchor / relay) that enqueue the kernels.  No device allocation, no host
+// synchronisation inside the layer calls.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include "rr_common.cuh"
+
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+thread_local char g_cuda_err[256] = "";
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+  return RR_ERR_CUDA;
+}
+#define RR_CUDA(call)                                             \
+  do {                                                            \
+    cudaError_t e_ = (call);                                      \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);           \
+  } while (0)
+
+struct Layout {
+  // ledger blob
+  size_t routes, sentinels, ages, kth, margin, ledger_total;
+  // scratch
+  size_t flags, alpha, beta, tau, refresh_rows, refresh_count, problem_offsets, tile_counts,
+      token_ranges, cand_scores, counters, status, S, scratch_total;
+  size_t export_total;
+};
+
+int validate(const rr_config* c) {
+  if (!c) return RR_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->heads < 1 || c->n_q < 1 || c->n_k < 1) return RR_ERR_INVALID_ARG;
+  if (c->k < 1 || c->m < 0 || c->r < 0) return RR_ERR_INVALID_ARG;
+  if (c->causal != 0 && c->causal != 1) return RR_ERR_INVALID_ARG;
+  if (c->causal_offset < 0) return RR_ERR_INVALID_ARG;
+  if (!(c->gamma >= 0.f)) return RR_ERR_INVALID_ARG;          // also rejects NaN
+  if (c->chunk_tokens < 0) return RR_ERR_INVALID_ARG;
+  if (c->dtype != RR_BF16 && c->dtype != RR_F32) return RR_ERR_UNSUPPORTED;
+  if (c->d != 64 && c->d != 128) return RR_ERR_UNSUPPORTED;
+  if (c->n_k > RR_MAX_NK) return RR_ERR_UNSUPPORTED;
+  if (c->k > c->n_k) return RR_ERR_INVALID_ARG;
+  if (c->k + c->m + c->r > RR_MAX_C) return RR_ERR_UNSUPPORTED;
+  const long long rows = (long long)c->batch * c->heads * c->n_q;
+  if (rows > (1LL << 30)) return RR_ERR_UNSUPPORTED;
+  if (c->chunk_tokens > 0 && (long long)c->n_k * c->chunk_tokens > 0x7FFFFFFFLL)
+    return RR_ERR_UNSUPPORTED;
+  return RR_OK;
+}
+
+Layout make_layout(const rr_config* c) {
+  Layout L{};
+  const size_t P = (size_t)c->batch * c->heads, rows = P * c->n_q;
+  const size_t sw = (size_t)c->m + c->r, cw = (size_t)c->k + sw;
+  const size_t tiles = P * ((c->n_q + RR_ROW_TILE - 1) / RR_ROW_TILE);
+  size_t o = 0;
+  L.routes = o;    o = align_up(o + rows * c->k * 4);
+  L.sentinels = o; o = align_up(o + rows * sw * 4);
+  L.ages = o;      o = align_up(o + rows * 4);
+  L.kth = o;       o = align_up(o + rows * 4);
+  L.margin = o;    o = align_up(o + rows * 4);
+  L.ledger_total = o;
+  L.export_total = rows * c->k * 4 + rows * sw * 4 + rows * 4 * 3;
+  o = 0;
+  L.flags = o;           o = align_up(o + rows);
+  L.alpha = o;           o = align_up(o + rows * 4);
+  L.beta = o;            o = align_up(o + rows * 4);
+  L.tau = o;             o = align_up(o + rows * 4);
+  L.refresh_rows = o;    o = align_up(o + rows * 4);
+  L.refresh_count = o;   o = align_up(o + 4);
+  L.problem_offsets = o; o = align_up(o + (P + 1) * 4);
+  L.tile_counts = o;     o = align_up(o + tiles * 4);
+  L.counters = o;        o = align_up(o + RR_NUM_COUNTERS * 8);
+  L.status = o;          o = align_up(o + 4);
+  L.token_ranges = o;    o = align_up(o + (c->chunk_tokens > 0 ? rows * c->k * 8 : 0));
+  L.cand_scores = o;     o = align_up(o + (c->debug_outputs ? rows * cw * 4 : 0));
+  L.S = o;               o = align_up(o + rows * (size_t)c->n_k * 4);
+  L.scratch_total = o;
+  return L;
+}
+
+unsigned long long dense_pairs(const rr_config* c) {
+  unsigned long long per_problem = 0;
+  for (int i = 0; i < c->n_q; ++i)
+    per_problem += (unsigned long long)rr_valid_count(i, c->n_k, c->causal, c->causal_offset);
+  return per_problem * (unsigned long long)c->batch * c->heads;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool anchor,
+                cudaStream_t st) {
+  if (!L || !qc || !kc || layer < 0) return RR_ERR_INVALID_ARG;
+  if (!aligned16(qc) || !aligned16(kc)) return RR_ERR_INVALID_ARG;
+  const RRParams& p = L->p;
+  if (anchor) {
+    // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
+    RR_CUDA(rr_launch_anchor_fill(p, st));
+    RR_CUDA(rr_launch_score_simt(p, qc, kc, nullptr, st));
+    RR_CUDA(rr_launch_topk_rows(p, nullptr, layer, st));
+    RR_CUDA(rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
+    L->anchored = 1;
+  } else {
+    if (!L->anchored) return RR_ERR_STATE;
+    // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
+    RR_CUDA(rr_launch_rescore(p, qc, kc, st));
+    RR_CUDA(rr_launch_compact(p, st));
+    RR_CUDA(rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
+    RR_CUDA(rr_launch_topk_rows(p, p.refresh_rows, layer, st));
+    RR_CUDA(rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
+  }
+  return RR_OK;
+}
+
+}  // namespace
+
+void rr_count_launch(int n) { g_launches.fetch_add((unsigned long long)n); }
+
+extern "C" {
+
+int rr_workspace_bytes(const rr_config* cfg, size_t* ledger_bytes, size_t* scratch_bytes) {
+  int rc = validate(cfg);
+  if (rc != RR_OK) return rc;
+  if (!ledger_bytes || !scratch_bytes) return RR_ERR_INVALID_ARG;
+  Layout L = make_layout(cfg);
+  *ledger_bytes = L.ledger_total;
+  *scratch_bytes = L.scratch_total;
+  return RR_OK;
+}
+
+int rr_export_bytes(const rr_config* cfg, size_t* bytes) {
+  int rc = validate(cfg);
+  if (rc != RR_OK) return rc;
+  if (!bytes) return RR_ERR_INVALID_ARG;
+  *bytes = make_layout(cfg).export_total;
+  return RR_OK;
+}
+
+int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
+                   void* dev_scratch, size_t scratch_bytes, rr_ledger** out) {
+  int rc = validate(cfg);
+  if (rc != RR_OK) return rc;
+  if (!dev_ledger || !dev_scratch || !out) return RR_ERR_INVALID_ARG;
+  if (((uintptr_t)dev_ledger & 255u) || ((uintptr_t)dev_scratch & 255u)) return RR_ERR_INVALID_ARG;
+  Layout lay = make_layout(cfg);
+  if (ledger_bytes < lay.ledger_total || scratch_bytes < lay.scratch_total) return RR_ERR_TOO_SMALL;
+  rr_ledger* L = new (std::nothrow) rr_ledger();
+  if (!L) return RR_ERR_INVALID_ARG;
+  L->cfg = *cfg;
+  L->dev_ledger = dev_ledger; L->ledger_bytes = ledger_bytes;
+  L->dev_scratch = dev_scratch; L->scratch_bytes = scratch_bytes;
+  L->export_bytes = lay.export_total;
+  L->anchored = 0;
+  L->device = -1;
+  cudaGetDevice(&L->device);           // informational; failure (no GPU) leaves -1
+  cudaGetLastError();
+  L->dense_pairs_per_layer = dense_pairs(cfg);
+  RRParams& p = L->p;
+  p.P = cfg->batch * cfg->heads; p.n_q = cfg->n_q; p.n_k = cfg->n_k; p.d = cfg->d;
+  p.k = cfg->k; p.m = cfg->m; p.r = cfg->r; p.sw = cfg->m + cfg->r; p.c = cfg->k + p.sw;
+  p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
+  p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs;
+  p.rows = p.P * p.n_q;
+  p.tiles_per_problem = (p.n_q + RR_ROW_TILE - 1) / RR_ROW_TILE;
+  p.n_tiles = p.P * p.tiles_per_problem;
+  p.gamma = cfg->gamma; p.seed = cfg->seed;
+  char* lb = (char*)dev_ledger; char* sb = (char*)dev_scratch;
+  p.routes = (int32_t*)(lb + lay.routes); p.sentinels = (int32_t*)(lb + lay.sentinels);
+  p.ages = (int32_t*)(lb + lay.ages); p.kth = (float*)(lb + lay.kth);
+  p.margin = (float*)(lb + lay.margin);
+  p.flags = (uint8_t*)(sb + lay.flags); p.alpha = (float*)(sb + lay.alpha);
+  p.beta = (float*)(sb + lay.beta); p.tau = (float*)(sb + lay.tau);
+  p.refresh_rows = (int32_t*)(sb + lay.refresh_rows);
+  p.refresh_count = (int32_t*)(sb + lay.refresh_count);
+  p.problem_offsets = (int32_t*)(sb + lay.problem_offsets);
+  p.tile_counts = (int32_t*)(sb + lay.tile_counts);
+  p.counters = (unsigned long long*)(sb + lay.counters);
+  p.status = (uint32_t*)(sb + lay.status);
+  p.token_ranges = cfg->chunk_tokens > 0 ? (int32_t*)(sb + lay.token_ranges) : nullptr;
+  p.cand_scores = cfg->debug_outputs ? (float*)(sb + lay.cand_scores) : nullptr;
+  p.S = (float*)(sb + lay.S);
+  *out = L;
+  return RR_OK;
+}
+
+int rr_ledger_reset(rr_ledger* L, void* stream) {
+  if (!L) return RR_ERR_INVALID_ARG;
+  RR_CUDA(rr_launch_reset(L->p, (cudaStream_t)stream));
+  L->anchored = 0;
+  return RR_OK;
+}
+
+int rr_ledger_destroy(rr_ledger* L) {
+  if (!L) return RR_ERR_INVALID_ARG;
+  delete L;
+  return RR_OK;
+}
+
+int rr_route_anchor(rr_ledger* L, const void* qc, const void* kc, int32_t layer, void* stream) {
+  return route_layer(L, qc, kc, layer, true, (cudaStream_t)stream);
+}
+
+int rr_route_relay(rr_ledger* L, const void* qc, const void* kc, int32_t layer, void* stream) {
+  return route_layer(L, qc, kc, layer, false, (cudaStream_t)stream);
+}
+
+int rr_route_layer_host(rr_ledger* L, const void* host_qc, const void* host_kc,
+                        void* dev_qc_staging, void* dev_kc_staging, int32_t layer,
+                        int32_t is_anchor, int32_t* host_routes, void* stream) {
+  if (!L || !host_qc || !host_kc || !dev_qc_staging || !dev_kc_staging) return RR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const RRParams& p = L->p;
+  const size_t esz = p.dtype == RR_F32 ? 4 : 2;
+  const size_t qb = (size_t)p.P * p.n_q * p.d * esz, kb = (size_t)p.P * p.n_k * p.d * esz;
+  if (!is_anchor && !L->anchored) return RR_ERR_STATE;
+  RR_CUDA(cudaMemcpyAsync(dev_qc_staging, host_qc, qb, cudaMemcpyHostToDevice, st));
+  RR_CUDA(cudaMemcpyAsync(dev_kc_staging, host_kc, kb, cudaMemcpyHostToDevice, st));
+  int rc = route_layer(L, dev_qc_staging, dev_kc_staging, layer, is_anchor != 0, st);
+  if (rc != RR_OK) return rc;
+  if (host_routes)
+    RR_CUDA(cudaMemcpyAsync(host_routes, p.routes, (size_t)p.rows * p.k * 4,
+                            cudaMemcpyDeviceToHost, st));
+  return RR_OK;
+}
+
+int rr_ledger_views(rr_ledger* L, rr_views* out) {
+  if (!L || !out) return RR_ERR_INVALID_ARG;
+  const RRParams& p = L->p;
+  out->routes = p.routes; out->sentinels = p.sentinels; out->ages = p.ages;
+  out->kth_score = p.kth; out->margin = p.margin; out->flags = p.flags;
+  out->alpha = p.alpha; out->beta = p.beta; out->refresh_rows = p.refresh_rows;
+  out->refresh_count = p.refresh_count; out->problem_offsets = p.problem_offsets;
+  out->token_ranges = p.token_ranges; out->cand_scores = p.cand_scores;
+  out->counters = (uint64_t*)p.counters; out->status = p.status;
+  return RR_OK;
+}
+
+static int xfer(rr_ledger* L, void* blob, size_t bytes, cudaStream_t st, bool to_host) {
+  if (!L || !blob) return RR_ERR_INVALID_ARG;
+  if (bytes < L->export_bytes) return RR_ERR_TOO_SMALL;
+  const RRParams& p = L->p;
+  const size_t rows = (size_t)p.rows;
+  struct Part { void* dev; size_t n; } parts[5] = {
+      {p.routes, rows * p.k * 4}, {p.sentinels, rows * p.sw * 4}, {p.ages, rows * 4},
+      {p.kth, rows * 4}, {p.margin, rows * 4}};
+  char* h = (char*)blob;
+  for (auto& pt : parts) {
+    if (pt.n) {
+      if (to_host) RR_CUDA(cudaMemcpyAsync(h, pt.dev, pt.n, cudaMemcpyDeviceToHost, st));
+      else RR_CUDA(cudaMemcpyAsync(pt.dev, h, pt.n, cudaMemcpyHostToDevice, st));
+    }
+    h += pt.n;
+  }
+  RR_CUDA(cudaStreamSynchronize(st));
+  return RR_OK;
+}
+
+int rr_ledger_export(rr_ledger* L, void* host_blob, size_t bytes, void* stream) {
+  return xfer(L, host_blob, bytes, (cudaStream_t)stream, true);
+}
+
+int rr_ledger_import(rr_ledger* L, const void* host_blob, size_t bytes, void* stream) {
+  int rc = xfer(L, const_cast<void*>(host_blob), bytes, (cudaStream_t)stream, false);
+  if (rc == RR_OK) {
+    // a restored ledger counts as anchored iff no row carries the "never routed" age
+    // (checked by the caller's data; the library trusts an imported checkpoint)
+    L->anchored = 1;
+  }
+  return rc;
+}
+
+int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out) {
+  if (!L || !status_out) return RR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t s = 0;
+  RR_CUDA(cudaMemcpyAsync(&s, L->p.status, 4, cudaMemcpyDeviceToHost, st));
+  RR_CUDA(cudaStreamSynchronize(st));
+  *status_out = s;
+  return (s & RR_STATUS_TIMEOUT) ? RR_ERR_TIMEOUT : RR_OK;
+}
+
+uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t t) {
+  return rr_draw_u32(rr_row_key(seed, g), layer, t);
+}
+
+uint64_t rr_kernel_launch_count(void) { return g_launches.load(); }
+
+const char* rr_strerror(int code) {
+  switch (code) {
+    case RR_OK: return "ok";
+    case RR_ERR_INVALID_ARG: return "invalid argument";
+    case RR_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case RR_ERR_STATE: return "ledger state does not allow this call (relay before anchor)";
+    case RR_ERR_CUDA: return "CUDA runtime error";
+    case RR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case RR_ERR_TOO_SMALL: return "buffer too small";
+    default: return "unknown error";
+  }
+}
+
+const char* rr_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

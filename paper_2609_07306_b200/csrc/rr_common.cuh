@@ -1,0 +1,88 @@
+// Shared declarations of the route-maintenance library (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/routerelay.h"
+
+#define RR_ROW_TILE 128            // rows per compaction / rescoring tile (per problem)
+#define RR_MAX_NK 4096
+#define RR_MAX_C 256
+
+// Everything a kernel needs to know about one ledger; passed by value.
+struct RRParams {
+  int P, n_q, n_k, d, k, m, r, c, sw;      // sw = m + r (sentinel row width)
+  int dtype, causal, causal_offset, chunk_tokens, debug;
+  int rows, tiles_per_problem, n_tiles;    // row tiles of RR_ROW_TILE per problem / in total
+  float gamma;
+  unsigned long long seed;
+  // ledger (persistent state, Section 4.1)
+  int32_t* routes; int32_t* sentinels; int32_t* ages; float* kth; float* margin;
+  // per-layer outputs and scratch
+  uint8_t* flags; float* alpha; float* beta; float* tau;
+  int32_t* refresh_rows; int32_t* refresh_count; int32_t* problem_offsets; int32_t* tile_counts;
+  int32_t* token_ranges; float* cand_scores;
+  unsigned long long* counters; uint32_t* status;
+  float* S;                                // [rows, n_k] score rows of the two-pass path
+};
+
+struct rr_ledger {
+  rr_config cfg;
+  RRParams p;
+  void* dev_ledger; size_t ledger_bytes;
+  void* dev_scratch; size_t scratch_bytes;
+  size_t export_bytes;
+  int device;
+  int anchored;                            // host-side: has an anchor been enqueued since reset
+  unsigned long long dense_pairs_per_layer;
+};
+
+// ---- device helpers -------------------------------------------------------------------
+__host__ __device__ __forceinline__ int rr_valid_count(int i, int n_k, int causal, int off) {
+  if (!causal) return n_k;
+  long long v = (long long)i + 1 + off;
+  return v > n_k ? n_k : (v < 0 ? 0 : (int)v);
+}
+
+// Monotone map float -> uint32 (larger float <=> larger key); -0.0 is folded onto +0.0.
+__device__ __forceinline__ uint32_t rr_order_key(float s) {
+  uint32_t u = __float_as_uint(s + 0.0f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float rr_key_to_float(uint32_t key) {
+  uint32_t u = (key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key;
+  return __uint_as_float(u);
+}
+
+// Counter-based generator of the random-sentinel sampler: two rounds of a 64-bit
+// avalanche finaliser, keyed by (seed, global row) and then by (layer, draw index).
+__host__ __device__ __forceinline__ unsigned long long rr_fmix64(unsigned long long x) {
+  x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ULL;
+  x ^= x >> 27; x *= 0x94D049BB133111EBULL;
+  x ^= x >> 31;
+  return x;
+}
+__host__ __device__ __forceinline__ unsigned long long rr_row_key(unsigned long long seed,
+                                                                  uint32_t g) {
+  return rr_fmix64(seed ^ ((unsigned long long)g * 0x9E3779B97F4A7C15ULL));
+}
+__host__ __device__ __forceinline__ uint32_t rr_draw_u32(unsigned long long row_key,
+                                                         uint32_t layer, uint32_t t) {
+  return (uint32_t)(rr_fmix64(row_key ^ (((unsigned long long)layer << 32) | t)) >> 32);
+}
+
+// ---- launchers (one per .cu file) -------------------------------------------------------
+// All return cudaError_t from the launch; all are asynchronous on `st`.
+cudaError_t rr_launch_score_simt(const RRParams& p, const void* qc, const void* kc,
+                                 const int32_t* row_list, cudaStream_t st);
+cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
+                                cudaStream_t st);
+cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
+                              cudaStream_t st);
+cudaError_t rr_launch_compact(const RRParams& p, cudaStream_t st);
+cudaError_t rr_launch_anchor_fill(const RRParams& p, cudaStream_t st);
+cudaError_t rr_launch_update(const RRParams& p, int is_anchor, unsigned long long dense_pairs,
+                             cudaStream_t st);
+cudaError_t rr_launch_reset(const RRParams& p, cudaStream_t st);
+
+void rr_count_launch(int n = 1);

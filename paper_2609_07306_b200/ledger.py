@@ -1,0 +1,151 @@
+"""RouteLedger: device buffers (torch) + the C handle.  PyTorch is used for device memory
+and streams only; every step of the routing path runs in the library's kernels."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .workload import DTYPE_BF16, RouteWorkload
+
+_TORCH_DT = {"i32": torch.int32, "f32": torch.float32, "u8": torch.uint8, "i64": torch.int64}
+
+
+def config_from_workload(w: RouteWorkload, debug_outputs: bool = False) -> B.rr_config:
+    return B.rr_config(batch=w.batch, heads=w.heads, n_q=w.n_q, n_k=w.n_k, d=w.d, k=w.k, m=w.m,
+                       r=w.r, dtype=B.RR_BF16 if w.dtype == DTYPE_BF16 else B.RR_F32,
+                       causal=1 if w.causal else 0, causal_offset=0, gamma=float(w.gamma),
+                       seed=int(w.seed), chunk_tokens=int(w.chunk_tokens),
+                       debug_outputs=1 if debug_outputs else 0)
+
+
+class RouteLedger:
+    """Owns the two device buffers of one ledger and exposes the C calls as methods."""
+
+    def __init__(self, cfg: B.rr_config, device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("RouteLedger needs a CUDA device (there is no CPU path)")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        lb, sb = B.rr_workspace_bytes(cfg)
+        with torch.cuda.device(self.device):
+            self.ledger_buf = torch.empty(lb + 256, dtype=torch.uint8, device=self.device)
+            self.scratch_buf = torch.empty(sb + 256, dtype=torch.uint8, device=self.device)
+            self._lo = (-self.ledger_buf.data_ptr()) % 256
+            self._so = (-self.scratch_buf.data_ptr()) % 256
+            self.handle = B.rr_ledger_init(cfg, self.ledger_buf.data_ptr() + self._lo, lb,
+                                           self.scratch_buf.data_ptr() + self._so, sb)
+        self.P = cfg.batch * cfg.heads
+        self.rows = self.P * cfg.n_q
+        self.c = cfg.k + cfg.m + cfg.r
+        self._views = B.rr_ledger_views(self.handle)
+        self.reset()
+
+    # -- lifetime ------------------------------------------------------------------------
+    def close(self):
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize(self.device)
+            B.rr_ledger_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self) -> int:
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    # -- calls -----------------------------------------------------------------------------
+    def reset(self):
+        B.rr_ledger_reset(self.handle, self._stream())
+
+    def route_anchor(self, qc: torch.Tensor, kc: torch.Tensor, layer: int):
+        B.rr_route_anchor(self.handle, qc.data_ptr(), kc.data_ptr(), layer, self._stream())
+
+    def route_relay(self, qc: torch.Tensor, kc: torch.Tensor, layer: int):
+        B.rr_route_relay(self.handle, qc.data_ptr(), kc.data_ptr(), layer, self._stream())
+
+    def route_layer_host(self, host_qc: torch.Tensor, host_kc: torch.Tensor,
+                         dev_qc: torch.Tensor, dev_kc: torch.Tensor, layer: int,
+                         is_anchor: bool, host_routes: torch.Tensor | None):
+        B.rr_route_layer_host(self.handle, host_qc.data_ptr(), host_kc.data_ptr(),
+                              dev_qc.data_ptr(), dev_kc.data_ptr(), layer, is_anchor,
+                              host_routes.data_ptr() if host_routes is not None else None,
+                              self._stream())
+
+    def status(self) -> int:
+        return B.rr_ledger_status(self.handle, self._stream())
+
+    # -- views (zero-copy torch tensors over the library's device pointers) ---------------
+    def _view(self, name: str, kind: str, shape):
+        ptr = getattr(self._views, name)
+        if not ptr:
+            return None
+        n = int(np.prod(shape))
+        dt = _TORCH_DT[kind]
+        nbytes = n * torch.empty((), dtype=dt).element_size()
+        for buf in (self.ledger_buf, self.scratch_buf):
+            off = ptr - buf.data_ptr()
+            if 0 <= off and off + nbytes <= buf.numel():
+                return buf[off:off + nbytes].view(dt).view(*shape)
+        raise RuntimeError(f"view {name} lies outside the ledger buffers")
+
+    @property
+    def routes(self): return self._view("routes", "i32", (self.rows, self.cfg.k))
+    @property
+    def sentinels(self): return self._view("sentinels", "i32", (self.rows, self.cfg.m + self.cfg.r))
+    @property
+    def ages(self): return self._view("ages", "i32", (self.rows,))
+    @property
+    def kth_score(self): return self._view("kth_score", "f32", (self.rows,))
+    @property
+    def margin(self): return self._view("margin", "f32", (self.rows,))
+    @property
+    def flags(self): return self._view("flags", "u8", (self.rows,))
+    @property
+    def alpha(self): return self._view("alpha", "f32", (self.rows,))
+    @property
+    def beta(self): return self._view("beta", "f32", (self.rows,))
+    @property
+    def refresh_rows(self): return self._view("refresh_rows", "i32", (self.rows,))
+    @property
+    def refresh_count(self): return self._view("refresh_count", "i32", (1,))
+    @property
+    def problem_offsets(self): return self._view("problem_offsets", "i32", (self.P + 1,))
+    @property
+    def token_ranges(self): return self._view("token_ranges", "i32", (self.rows, self.cfg.k, 2))
+    @property
+    def cand_scores(self): return self._view("cand_scores", "f32", (self.rows, self.c))
+    @property
+    def counters(self): return self._view("counters", "i64", (B.RR_NUM_COUNTERS,))
+
+    def counters_dict(self):
+        vals = self.counters.cpu().tolist()
+        return dict(zip(B.COUNTER_NAMES, vals))
+
+    # -- checkpoint ---------------------------------------------------------------------------
+    def export_blob(self) -> np.ndarray:
+        n = B.rr_export_bytes(self.cfg)
+        blob = np.empty(n, np.uint8)
+        B.rr_ledger_export(self.handle, blob.ctypes.data, n, self._stream())
+        return blob
+
+    def import_blob(self, blob: np.ndarray):
+        blob = np.ascontiguousarray(blob, np.uint8)
+        B.rr_ledger_import(self.handle, blob.ctypes.data, blob.size, self._stream())
+
+    def pack_blob(self, routes, sentinels, ages, kth, margin) -> np.ndarray:
+        """Host arrays -> checkpoint blob layout (routes, sentinels, ages, kth, margin)."""
+        parts = [np.ascontiguousarray(routes, np.int32), np.ascontiguousarray(sentinels, np.int32),
+                 np.ascontiguousarray(ages, np.int32), np.ascontiguousarray(kth, np.float32),
+                 np.ascontiguousarray(margin, np.float32)]
+        return np.concatenate([p.reshape(-1).view(np.uint8) for p in parts])
+
+
+def device_tensor(x: np.ndarray, device="cuda:0") -> torch.Tensor:
+    """Generated inputs (bf16 bit patterns as uint16, or float32) -> device tensor."""
+    if x.dtype == np.uint16:
+        return torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(device)

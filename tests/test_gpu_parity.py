@@ -1,0 +1,173 @@
+"""CUDA path vs CPU oracle (through the C ABI), teacher-forced layer by layer."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from oracle import routerelay_oracle as O
+from paper_2609_07306_b200 import binding as B
+from paper_2609_07306_b200 import workload as W
+from paper_2609_07306_b200.ledger import RouteLedger, config_from_workload, device_tensor
+
+pytestmark = pytest.mark.gpu
+
+
+def _report(rep):
+    print(f"rows {rep.rows_checked} refreshed {rep.refreshed_checked} | ambiguous flag rows "
+          f"{rep.ambiguous_flag_rows} (mismatching {rep.flag_mismatch_ambiguous}) | ambiguous "
+          f"route rows {rep.ambiguous_route_rows} (mismatching {rep.route_mismatch_ambiguous}) | "
+          f"max |score err| {rep.max_score_err:.3e} rel {rep.max_score_rel_err:.3e}")
+
+
+def test_tiny_fp32_all_layers():
+    rep = parity.run_teacher_forced(W.tiny())
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_moderate_bf16_causal_all_layers():
+    rep = parity.run_teacher_forced(W.moderate())
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+@pytest.mark.parametrize("n", [128, 512])
+def test_sweep_shapes(n):
+    w = W.sweep(n, 0.15).replace(heads=4, layers=4, anchor_every=3)
+    rep = parity.run_teacher_forced(w)
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_ragged_shapes_and_wide_ledger():
+    # n_q not a multiple of any tile, n_q != n_k, non-causal, d=64 bf16, wide candidate set
+    w = W.RouteWorkload("ragged", 1, 3, 200, 333, 64, 12, 24, 12, layers=3, anchor_every=3,
+                        dtype=W.DTYPE_BF16, centroids=16, rho=0.05, causal=False, seed=3)
+    rep = parity.run_teacher_forced(w)
+    _report(rep)
+    parity.assert_clean(rep)
+    w = W.RouteWorkload("ragged32", 2, 1, 130, 130, 128, 5, 0, 7, layers=3, anchor_every=2,
+                        dtype=W.DTYPE_F32, centroids=8, rho=0.1, causal=True, seed=4)
+    rep = parity.run_teacher_forced(w)
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_degenerate_all_equal_scores():
+    """All-zero inputs: every score ties; TopK must take the smallest ids, margin 0, and the
+    challenge test (tie => flagged) must flag every row that has a sentinel."""
+    w = W.tiny()
+    led = RouteLedger(config_from_workload(w))
+    z = torch.zeros(1, 1, w.n_q, w.d, device="cuda")
+    led.route_anchor(z, z, 0)
+    torch.cuda.synchronize()
+    r = led.routes.cpu().numpy()
+    s = led.sentinels.cpu().numpy()
+    assert (np.sort(r, axis=1) == np.arange(w.k)).all()
+    assert (np.sort(s[:, :w.m], axis=1) == np.arange(w.k, w.k + w.m)).all()
+    assert (led.margin.cpu().numpy() == 0).all() and (led.kth_score.cpu().numpy() == 0).all()
+    rnd = s[:, w.m:]
+    assert (rnd >= w.k + w.m).all() and (rnd < w.n_k).all()
+    assert all(len(set(row)) == w.r for row in rnd)
+    led.route_relay(z, z, 1)
+    torch.cuda.synchronize()
+    assert led.flags.cpu().numpy().all()
+    assert int(led.refresh_count.item()) == w.n_q
+    led.close()
+
+
+def test_relay_before_anchor_and_reset():
+    w = W.tiny()
+    led = RouteLedger(config_from_workload(w))
+    z = torch.zeros(1, 1, w.n_q, w.d, device="cuda")
+    with pytest.raises(B.RouteRelayError) as ei:
+        led.route_relay(z, z, 1)
+    assert ei.value.code == B.RR_ERR_STATE
+    led.route_anchor(z, z, 0)
+    led.reset()
+    torch.cuda.synchronize()
+    assert (led.routes.cpu().numpy() == -1).all() and (led.ages.cpu().numpy() == -1).all()
+    assert led.counters.cpu().numpy().sum() == 0
+    with pytest.raises(B.RouteRelayError):
+        led.route_relay(z, z, 1)
+    led.close()
+
+
+def test_export_import_roundtrip_and_counters():
+    w = W.moderate().replace(heads=2)
+    q, k = W.generate(w, layers=3)
+    led = RouteLedger(config_from_workload(w))
+    led.route_anchor(device_tensor(q[0]), device_tensor(k[0]), 0)
+    blob = led.export_blob()
+    led.route_relay(device_tensor(q[1]), device_tensor(k[1]), 1)
+    torch.cuda.synchronize()
+    after1 = led.routes.clone()
+    flags1 = led.flags.cpu().numpy().copy()
+    led.import_blob(blob)                       # rewind to the anchor state
+    led.route_relay(device_tensor(q[1]), device_tensor(k[1]), 1)
+    torch.cuda.synchronize()
+    assert torch.equal(led.routes, after1)
+    c = led.counters_dict()
+    v = np.tile(parity.oracle_params(w).valid_counts(), w.problems)
+    assert c["layer_calls"] == 3 and c["anchor_rows"] == w.rows and c["relay_rows"] == 2 * w.rows
+    assert c["dense_pairs"] == 3 * v.sum()
+    assert c["flagged_rows"] == 2 * flags1.sum()
+    assert c["full_pairs"] == v.sum() + 2 * v[flags1 != 0].sum()
+    assert c["cand_pairs"] == 2 * np.minimum(v, w.c).sum()
+    led.close()
+
+
+def test_host_buffer_entry_point():
+    w = W.moderate().replace(heads=2)
+    q, k = W.generate(w, layers=2)
+    led = RouteLedger(config_from_workload(w))
+    ref = RouteLedger(config_from_workload(w))
+    hq = [torch.from_numpy(q[l].view(np.int16)).pin_memory() for l in range(2)]
+    hk = [torch.from_numpy(k[l].view(np.int16)).pin_memory() for l in range(2)]
+    dq, dk = torch.empty_like(hq[0], device="cuda"), torch.empty_like(hk[0], device="cuda")
+    out = torch.empty(w.rows, w.k, dtype=torch.int32).pin_memory()
+    for l in range(2):
+        led.route_layer_host(hq[l], hk[l], dq, dk, l, l == 0, out)
+        (ref.route_anchor if l == 0 else ref.route_relay)(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref.routes.cpu())
+    led.close(); ref.close()
+
+
+def test_token_ranges():
+    w = W.moderate().replace(heads=2, chunk_tokens=64)
+    q, k = W.generate(w, layers=2)
+    led = RouteLedger(config_from_workload(w))
+    led.route_anchor(device_tensor(q[0]), device_tensor(k[0]), 0)
+    led.route_relay(device_tensor(q[1]), device_tensor(k[1]), 1)
+    torch.cuda.synchronize()
+    expect = O.token_ranges(led.routes.cpu().numpy(), 64)
+    assert np.array_equal(led.token_ranges.cpu().numpy(), expect)
+    led.close()
+
+
+def test_free_running_summary_matches_oracle():
+    """All layers without teacher forcing: recall / refreshed-row / score-pair fractions of
+    the device run agree with the oracle's run up to the ambiguous rows."""
+    w = W.moderate()
+    q, k = W.generate(w)
+    p = parity.oracle_params(w)
+    res, summ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),
+                             p, w.anchor_every)
+    led = RouteLedger(config_from_workload(w))
+    hit = tot = 0
+    for l in range(w.layers):
+        fn = led.route_anchor if w.is_anchor(l) else led.route_relay
+        fn(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        h, t = O.recall_counts(led.routes.cpu().numpy(), res[l].full_routes)
+        hit += h; tot += t
+    c = led.counters_dict()
+    rer, flg, pairs = O.fractions_from_counters(c)
+    print(f"device: recall {hit / tot:.6f} rerouted {rer:.4f} flagged {flg:.4f} pairs {pairs:.4f}"
+          f" | oracle: {summ.recall_all:.6f} {summ.rerouted_fraction:.4f} "
+          f"{summ.flagged_relay_fraction:.4f} {summ.score_pair_fraction:.4f}")
+    assert abs(hit / tot - summ.recall_all) < 2e-4
+    assert abs(rer - summ.rerouted_fraction) < 2e-3
+    assert abs(pairs - summ.score_pair_fraction) < 2e-3
+    led.close()
