@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the route-maintenance hot path (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload high_drift]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+A step is one pass of the whole hot path over one batch of synthetic input: every layer
+of the workload's schedule (anchor layers: score GEMM + TopK + sentinel build; relay layers:
+candidate rescoring, challenge test, compaction, row-selective refresh, ledger update).
+`value` = query rows routed per second per layer = rows * layers * n_gpus / time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_07306_b200 import workload as W  # noqa: E402
+
+METRIC = "layer-route rows/sec per layer (n_k=1024) vs full GEMM+TopK routing"
+UNIT = "rows/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+def _workload(name: str) -> W.RouteWorkload:
+    if name == "sweep1024":
+        return W.sweep(1024, 0.30)
+    return W.PRESETS[name]()
+
+
+# ----------------------------------------------------------------------------- reference arm
+def _oracle_sample(w: W.RouteWorkload, n_problems: int, n_layers: int):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload."""
+    from oracle import routerelay_oracle as O
+    problems = list(range(min(n_problems, w.problems)))
+    n_layers = min(n_layers, w.layers)
+    q, k = W.generate(w, problems=problems, layers=n_layers)
+    qf = W.as_float32(q).astype(np.float64)
+    kf = W.as_float32(k).astype(np.float64)
+    p = O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, gamma=w.gamma, causal=w.causal,
+                       causal_offset=0, seed=w.seed)
+    t0 = time.perf_counter()
+    _, summ = O.run_layers(qf, kf, p, w.anchor_every, problems)
+    dt = time.perf_counter() - t0
+    rows = len(problems) * w.n_q * n_layers
+    return rows / dt, dt, summ, f"{len(problems)} of {w.problems} problems x first {n_layers} of " \
+                                f"{w.layers} layers ({rows} row-layers, {dt:.1f} s)"
+
+
+def _blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([int(i.get("num_threads", 1)) for i in threadpool_info()] or [1])
+    except Exception:
+        return 1
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = _workload(args.workload)
+    vals = []
+    sample = ""
+    for s in range(args.warmup + args.steps):
+        v, dt, summ, sample = _oracle_sample(w, 2, 5)
+        if s >= args.warmup:
+            vals.append((v, dt))
+    value = sum(v for v, _ in vals) / len(vals)
+    ms = 1e3 * sum(dt for _, dt in vals) / len(vals)
+    cores = _blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample_per_step": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(gpu_index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- roofline
+def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
+    """Algorithmic work of one kernel kind over one step, its bound and measured peak.
+
+    cnt: work counters of one step (anchor_rows, relay_rows, flagged_rows, cand_pairs,
+    full_pairs).  Figures per unit are spelled out in the design doc."""
+    esz = 2 if w.dtype == W.DTYPE_BF16 else 4
+    routed = cnt["anchor_rows"] + cnt["flagged_rows"]
+    layer_calls = cnt["layer_calls"]
+    n_anchor = cnt["anchor_rows"] // w.rows
+    in_bytes = w.problems * (w.n_q + w.n_k) * w.d * esz
+    ledger_row = (w.c + 2) * 4
+    sec = ms * 1e-3
+    if kind == "topk_rows":        # reads score rows, writes ledger rows
+        alg = cnt["full_pairs"] * 4 + routed * ledger_row
+        return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                    alg_per_launch=alg / launches)
+    if kind == "rescore":          # unique bytes: inputs + ledger ids + flags/alpha/beta
+        alg = (layer_calls - n_anchor) * (in_bytes + w.rows * (w.c * 4 + 9))
+        return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                    alg_per_launch=alg / launches)
+    if kind == "score_simt":       # fp32 FMA: 2*d flop per score pair
+        alg = 2.0 * w.d * cnt["full_pairs"]
+        mhz = sm_mhz or 1965.0
+        peak = 148 * 128 * 2 * mhz * 1e6 / 1e12
+        return dict(bound="alu", achieved=alg / sec / 1e12, peak=peak, unit="TFLOP/s",
+                    alg_per_launch=alg / launches)
+    if kind in ("score_tc", "route_fused"):
+        alg = 2.0 * w.d * cnt["full_pairs"]
+        return dict(bound="tensor", achieved=alg / sec / 1e12,
+                    peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                    alg_per_launch=alg / launches)
+    if kind == "compact":
+        alg = (layer_calls - n_anchor) * w.rows + cnt["flagged_rows"] * 4
+        return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                    alg_per_launch=alg / launches)
+    alg = layer_calls * w.rows * 9
+    return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                alg_per_launch=alg / launches)
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args) -> None:
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_07306_b200 import binding as B
+    from paper_2609_07306_b200.ledger import RouteLedger, config_from_workload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path "
+                         "(use --impl reference for the CPU oracle)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    w = _workload(args.workload).replace(seed=rank)      # weak scaling: own problems per rank
+    L = w.layers
+    peaks = _peaks()
+    esz = 2 if w.dtype == W.DTYPE_BF16 else 4
+    tdt = torch.int16 if w.dtype == W.DTYPE_BF16 else torch.float32
+    ndt = np.uint16 if w.dtype == W.DTYPE_BF16 else np.float32
+
+    # ---- inputs: generated on the host into pinned memory, then staged to the device -----
+    t_gen = time.perf_counter()
+    hq = torch.empty((L, w.problems, w.n_q, w.d), dtype=tdt).pin_memory()
+    hk = torch.empty((L, w.problems, w.n_k, w.d), dtype=tdt).pin_memory()
+    W.generate(w, threads=max(1, (os.cpu_count() or 8) // max(1, world)),
+               out_q=hq.numpy().view(ndt), out_k=hk.numpy().view(ndt))
+    t_gen = time.perf_counter() - t_gen
+    dq, dk = hq.to(dev), hk.to(dev)
+    if w.dtype == W.DTYPE_BF16:
+        dq, dk = dq.view(torch.bfloat16), dk.view(torch.bfloat16)
+
+    led = RouteLedger(config_from_workload(w), device=str(dev))
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        for l in range(L):
+            if w.is_anchor(l):
+                led.route_anchor(dq[l], dk[l], l)
+            else:
+                led.route_relay(dq[l], dk[l], l)
+
+    # ---- timed region: device-resident inputs ----------------------------------------------
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    clocks = ClockSampler(local)
+    launches0 = B.rr_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    launches = B.rr_kernel_launch_count() - launches0
+    clock_info = clocks.stop()
+    ms_per_step = ms_total / args.steps
+    value = w.rows * L * world / (ms_per_step * 1e-3)
+
+    # ---- per-kernel device times (same steps, events around every launch) ---------------
+    led.reset()
+    B.rr_profile_begin(led.handle)
+    for _ in range(args.steps):
+        step()
+    prof = B.rr_profile_end(led.handle, stream.cuda_stream)
+    cnt = {k: v // args.steps for k, v in led.counters_dict().items()}
+    tot_ms = sum(ms for ms, _ in prof.values())
+    kernels = {}
+    for kind, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0]):
+        r = _kernel_roofline(kind, ms / args.steps, n / args.steps, w, cnt, peaks,
+                             clock_info.get("sm_mhz"))
+        kernels[kind] = {"launches_per_step": n // args.steps, "avg_us": 1e3 * ms / n,
+                         "share": ms / tot_ms, "bound": r["bound"], "achieved": r["achieved"],
+                         "peak": r["peak"], "unit": r["unit"], "frac": r["achieved"] / r["peak"]}
+    top = next(iter(kernels))
+    tk = kernels[top]
+    roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
+                "peak": tk["peak"], "unit": tk["unit"], "frac": tk["frac"],
+                "peak_source": peaks["source"] if tk["bound"] != "alu" else
+                "148 SMs x 128 FMA/clk x 2 x sampled SM clock", "traffic": None}
+
+    # ---- per-layer times: anchor layers, relay layers, and full routing on every layer ---
+    def per_layer_ms(fn_of_layer):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(L + 1)]
+        ev[0].record(stream)
+        for l in range(L):
+            fn_of_layer(l)
+            ev[l + 1].record(stream)
+        torch.cuda.synchronize()
+        return [ev[l].elapsed_time(ev[l + 1]) for l in range(L)]
+
+    def sched(l):
+        (led.route_anchor if w.is_anchor(l) else led.route_relay)(dq[l], dk[l], l)
+
+    reps = [per_layer_ms(sched) for _ in range(3)]
+    layer_ms = [statistics.median(r[l] for r in reps) for l in range(L)]
+    anchor_ms = statistics.median(layer_ms[l] for l in range(L) if w.is_anchor(l))
+    relay_ms = statistics.median(layer_ms[l] for l in range(L) if not w.is_anchor(l))
+    full_led = RouteLedger(config_from_workload(w), device=str(dev))
+    freps = [per_layer_ms(lambda l: full_led.route_anchor(dq[l], dk[l], l)) for _ in range(3)]
+    full_ms = statistics.median(statistics.median(r[l] for r in freps) for l in range(L))
+
+    # ---- quality: recall vs full routing, refreshed-row and score-pair fractions -----------
+    led.reset()
+    hit = tot = 0
+    for l in range(L):
+        sched(l)
+        full_led.route_anchor(dq[l], dk[l], l)
+        a, b = led.routes, full_led.routes
+        for lo in range(0, w.rows, 65536):
+            aa, bb = a[lo:lo + 65536], b[lo:lo + 65536]
+            inter = ((aa.unsqueeze(2) == bb.unsqueeze(1)) & (bb.unsqueeze(1) >= 0)).any(2)
+            hit += int(inter.sum().item())
+            tot += int((bb >= 0).sum().item())
+    c1 = led.counters_dict()
+    rerouted = (c1["anchor_rows"] + c1["flagged_rows"]) / (c1["anchor_rows"] + c1["relay_rows"])
+    flagged = c1["flagged_rows"] / max(1, c1["relay_rows"])
+    pairs = (c1["cand_pairs"] + c1["full_pairs"]) / c1["dense_pairs"]
+    status = led.status()
+
+    # ---- end to end: host buffers through rr_route_layer_host --------------------------------
+    sq = torch.empty_like(dq[0]); sk = torch.empty_like(dk[0])
+    host_routes = torch.empty((w.rows, w.k), dtype=torch.int32).pin_memory()
+
+    def step_e2e():
+        for l in range(L):
+            led.route_layer_host(hq[l], hk[l], sq, sk, l, w.is_anchor(l), host_routes)
+
+    step_e2e()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record(stream)
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    h2d = L * w.problems * (w.n_q + w.n_k) * w.d * esz
+    d2h = L * w.rows * w.k * 4
+    e2e = {"value": w.rows * L * world / (ms_e2e * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only) -----------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, dt, summ, sample = _oracle_sample(w, 4, 9)
+        cpu = {"value": v, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+               "sample": sample, "oracle_recall": summ.recall_all,
+               "oracle_flagged_fraction": summ.flagged_relay_fraction}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == W.DTYPE_BF16 else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "problems": w.problems, "n_q": w.n_q, "n_k": w.n_k,
+                       "d": w.d, "k": w.k, "m": w.m, "r": w.r, "layers": L,
+                       "anchor_every": w.anchor_every, "rho": w.rho, "causal": w.causal,
+                       "l2": "inputs of consecutive layers differ and exceed L2 "
+                             f"({w.problems * (w.n_q + w.n_k) * w.d * esz / 1e6:.0f} MB/layer)",
+                       "host_generation_s": round(t_gen, 1)},
+            "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+            "layers": {"anchor_ms": anchor_ms, "relay_ms": relay_ms, "full_routing_ms": full_ms,
+                       "anchor_rows_per_s": w.rows / anchor_ms * 1e3,
+                       "relay_rows_per_s": w.rows / relay_ms * 1e3,
+                       "full_routing_rows_per_s": w.rows / full_ms * 1e3,
+                       "relay_speedup_vs_full": full_ms / relay_ms},
+            "quality": {"recall_vs_full_routing": hit / tot, "rerouted_row_fraction": rerouted,
+                        "flagged_relay_row_fraction": flagged, "score_pair_fraction": pairs,
+                        "status_word": status},
+            "kernels": kernels,
+        }
+        print(json.dumps(line))
+    led.close(); full_led.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="high_drift",
+                    choices=sorted(W.PRESETS) + ["sweep1024"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

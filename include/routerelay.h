@@ -157,6 +157,25 @@ int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out);
  * global row g when its sentinels are rebuilt at `layer`); same code the kernels run. */
 uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t t);
 
+/* Per-kernel device timing for benchmarks.  Between rr_profile_begin and rr_profile_end
+ * every kernel the layer calls launch is bracketed by CUDA events on the caller's stream
+ * (this adds event records to the stream; do not leave it on in production).
+ * rr_profile_end synchronises the stream and returns, per kernel kind (RR_KIND_*), the total
+ * device time in milliseconds and the number of launches; arrays hold RR_NUM_KINDS entries. */
+#define RR_KIND_SCORE_SIMT   0   /* score rows on FP32 ALUs (fp32 inputs)                    */
+#define RR_KIND_TOPK_ROWS    1   /* warp-level TopK + sentinels over score rows in memory    */
+#define RR_KIND_RESCORE      2   /* gathered candidate rescoring + challenge test            */
+#define RR_KIND_COMPACT      3   /* ballot / prefix-scan row compaction                      */
+#define RR_KIND_ANCHOR_FILL  4   /* anchor: flags, identity refresh list                     */
+#define RR_KIND_UPDATE       5   /* ledger update: ages, counters                            */
+#define RR_KIND_EXPAND       6   /* token-range expansion                                    */
+#define RR_KIND_SCORE_TC     7   /* tcgen05 score GEMM                                       */
+#define RR_KIND_ROUTE_FUSED  8   /* tcgen05 score GEMM fused with TopK + sentinels           */
+#define RR_NUM_KINDS        12
+int rr_profile_begin(rr_ledger* L);
+int rr_profile_end(rr_ledger* L, void* stream, float* total_ms, int64_t* launches);
+const char* rr_kind_name(int kind);
+
 /* How many kernels the library has launched since it was loaded (all ledgers). */
 uint64_t rr_kernel_launch_count(void);
 

@@ -25,6 +25,7 @@ RR_STATUS_TIMEOUT = 1
 RR_STATUS_BAD_INDEX = 2
 RR_STATUS_OVERFLOW = 4
 RR_NUM_COUNTERS = 8
+RR_NUM_KINDS = 12
 COUNTER_NAMES = ("layer_calls", "anchor_rows", "relay_rows", "flagged_rows", "cand_pairs",
                  "full_pairs", "dense_pairs")
 
@@ -81,6 +82,12 @@ def lib() -> C.CDLL:
         L.rr_ledger_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
         L.rr_sampler_draw_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
         L.rr_sampler_draw_u32.restype = C.c_uint32
+        L.rr_profile_begin.argtypes = [vp]
+        L.rr_profile_begin.restype = C.c_int
+        L.rr_profile_end.argtypes = [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+        L.rr_profile_end.restype = C.c_int
+        L.rr_kind_name.argtypes = [C.c_int]
+        L.rr_kind_name.restype = C.c_char_p
         L.rr_kernel_launch_count.argtypes = []
         L.rr_kernel_launch_count.restype = C.c_uint64
         L.rr_strerror.argtypes = [C.c_int]
@@ -174,6 +181,22 @@ def rr_ledger_status(h: int, stream: int) -> int:
 
 def rr_sampler_draw_u32(seed: int, g: int, layer: int, t: int) -> int:
     return int(lib().rr_sampler_draw_u32(seed, g, layer, t))
+
+
+def rr_profile_begin(h: int) -> None:
+    _check(lib().rr_profile_begin(h), "rr_profile_begin")
+
+
+def rr_profile_end(h: int, stream: int):
+    """{kind name: (total ms, launches)} for the kinds that ran."""
+    ms = (C.c_float * RR_NUM_KINDS)()
+    n = (C.c_int64 * RR_NUM_KINDS)()
+    _check(lib().rr_profile_end(h, stream, ms, n), "rr_profile_end")
+    out = {}
+    for i in range(RR_NUM_KINDS):
+        if n[i]:
+            out[lib().rr_kind_name(i).decode()] = (float(ms[i]), int(n[i]))
+    return out
 
 
 def rr_kernel_launch_count() -> int:

@@ -99,22 +99,34 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   if (!L || !qc || !kc || layer < 0) return RR_ERR_INVALID_ARG;
   if (!aligned16(qc) || !aligned16(kc)) return RR_ERR_INVALID_ARG;
   const RRParams& p = L->p;
+  // LAUNCH(kind, call): enqueue one kernel, bracketed by events while profiling
+#define LAUNCH(kind, call)                                                         \
+  do {                                                                             \
+    rr_ledger::ProfRec rec_{kind, nullptr, nullptr};                               \
+    if (L->profiling) {                                                            \
+      RR_CUDA(cudaEventCreate(&rec_.a)); RR_CUDA(cudaEventCreate(&rec_.b));        \
+      RR_CUDA(cudaEventRecord(rec_.a, st));                                        \
+    }                                                                              \
+    RR_CUDA(call);                                                                 \
+    if (L->profiling) { RR_CUDA(cudaEventRecord(rec_.b, st)); L->prof.push_back(rec_); } \
+  } while (0)
   if (anchor) {
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
-    RR_CUDA(rr_launch_anchor_fill(p, st));
-    RR_CUDA(rr_launch_score_simt(p, qc, kc, nullptr, st));
-    RR_CUDA(rr_launch_topk_rows(p, nullptr, layer, st));
-    RR_CUDA(rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
+    LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, st));
+    LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
+    LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, nullptr, layer, st));
+    LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
     L->anchored = 1;
   } else {
     if (!L->anchored) return RR_ERR_STATE;
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
-    RR_CUDA(rr_launch_rescore(p, qc, kc, st));
-    RR_CUDA(rr_launch_compact(p, st));
-    RR_CUDA(rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
-    RR_CUDA(rr_launch_topk_rows(p, p.refresh_rows, layer, st));
-    RR_CUDA(rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
+    LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
+    LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, st));
+    LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
+    LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, p.refresh_rows, layer, st));
+    LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
   }
+#undef LAUNCH
   return RR_OK;
 }
 
@@ -287,6 +299,45 @@ int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out) {
 
 uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t t) {
   return rr_draw_u32(rr_row_key(seed, g), layer, t);
+}
+
+int rr_profile_begin(rr_ledger* L) {
+  if (!L) return RR_ERR_INVALID_ARG;
+  for (auto& r : L->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  L->prof.clear();
+  L->profiling = true;
+  return RR_OK;
+}
+
+int rr_profile_end(rr_ledger* L, void* stream, float* total_ms, int64_t* launches) {
+  if (!L || !total_ms || !launches) return RR_ERR_INVALID_ARG;
+  L->profiling = false;
+  for (int i = 0; i < RR_NUM_KINDS; ++i) { total_ms[i] = 0.f; launches[i] = 0; }
+  RR_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  for (auto& r : L->prof) {
+    float ms = 0.f;
+    RR_CUDA(cudaEventElapsedTime(&ms, r.a, r.b));
+    total_ms[r.kind] += ms;
+    launches[r.kind] += 1;
+    cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+  }
+  L->prof.clear();
+  return RR_OK;
+}
+
+const char* rr_kind_name(int kind) {
+  switch (kind) {
+    case RR_KIND_SCORE_SIMT: return "score_simt";
+    case RR_KIND_TOPK_ROWS: return "topk_rows";
+    case RR_KIND_RESCORE: return "rescore";
+    case RR_KIND_COMPACT: return "compact";
+    case RR_KIND_ANCHOR_FILL: return "anchor_fill";
+    case RR_KIND_UPDATE: return "update";
+    case RR_KIND_EXPAND: return "expand";
+    case RR_KIND_SCORE_TC: return "score_tc";
+    case RR_KIND_ROUTE_FUSED: return "route_fused";
+    default: return "";
+  }
 }
 
 uint64_t rr_kernel_launch_count(void) { return g_launches.load(); }

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <vector>
 #include "../../include/routerelay.h"
 
 #define RR_ROW_TILE 128            // rows per compaction / rescoring tile (per problem)
@@ -35,6 +36,10 @@ struct rr_ledger {
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
   unsigned long long dense_pairs_per_layer;
+  // benchmark-only per-kernel timing
+  bool profiling = false;
+  struct ProfRec { int kind; cudaEvent_t a, b; };
+  std::vector<ProfRec> prof;
 };
 
 // ---- device helpers -------------------------------------------------------------------
