@@ -50,6 +50,7 @@ extern "C" {
 #define RR_ERR_CUDA          -4   /* a CUDA runtime call failed (see rr_last_cuda_error)       */
 #define RR_ERR_TIMEOUT       -5   /* a bounded device-side wait expired (device status word)   */
 #define RR_ERR_TOO_SMALL     -6   /* caller-provided buffer smaller than required              */
+#define RR_ERR_TOO_LARGE     -7   /* problem exceeds a fixed built-in capacity                 */
 
 #define RR_BF16 0
 #define RR_F32  1
@@ -156,6 +157,38 @@ int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out);
 /* Host-callable copy of the sampler's counter-based generator (the t-th 32-bit draw of
  * global row g when its sentinels are rebuilt at `layer`); same code the kernels run. */
 uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t t);
+
+/* Row compaction for callers that cannot allocate device memory.  (The paper has no
+ * counterpart of this entry point; it computes the same list as the compaction step of
+ * rr_route_relay, Section 4.2.)
+ *
+ * Who needs it: code that runs where cudaMalloc may not be called -- a serving process
+ * whose device memory pool is frozen after start-up, a plugin that is handed its input
+ * and output buffers and nothing more, a latency path that cannot afford the implicit
+ * synchronisation of an allocation.  The ledger API above asks such a caller for a scratch
+ * buffer; this call asks for nothing beyond inputs and outputs.  Its scratch (per-tile
+ * flagged counts) lives in a fixed array inside the library image: every GPU that loads
+ * the library holds RR_NOALLOC_MAX_TILES * 4 bytes (256 KB) for it until the process exits.
+ *
+ *   dev_flags               [n_problems * n_q] device, in : non-zero = row is flagged
+ *   dev_rows_out            [n_problems * n_q] device, out: ascending global ids of the flagged
+ *                           rows in the first *dev_count_out entries (rest untouched)
+ *   dev_count_out           [1] device, out
+ *   dev_problem_offsets_out [n_problems + 1] device, out: exclusive scan of per-problem counts
+ *
+ * Limit: ceil(n_q / 128) * n_problems <= RR_NOALLOC_MAX_TILES (8.4 M rows when n_q is a
+ * multiple of 128); larger inputs return RR_ERR_TOO_LARGE and nothing is enqueued.
+ * The call allocates nothing, on the host or the device, and only enqueues work on `stream`.
+ * The first call on a device also looks up the array's device address (once per device,
+ * with that device current); make that first call before starting any stream capture.
+ * All calls share the one array, which keeps the previous call's contents (every entry
+ * that is read is rewritten first, so nothing needs clearing): calls whose kernels can
+ * overlap on the GPU -- different streams or threads -- race and must be serialised by
+ * the caller. */
+#define RR_NOALLOC_MAX_TILES 65536
+int rr_compact_flags_noalloc(const uint8_t* dev_flags, int32_t n_problems, int32_t n_q,
+                             int32_t* dev_rows_out, int32_t* dev_count_out,
+                             int32_t* dev_problem_offsets_out, void* stream);
 
 /* Per-kernel device timing for benchmarks.  Between rr_profile_begin and rr_profile_end
  * every kernel the layer calls launch is bracketed by CUDA events on the caller's stream

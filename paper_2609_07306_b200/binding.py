@@ -19,6 +19,8 @@ RR_ERR_STATE = -3
 RR_ERR_CUDA = -4
 RR_ERR_TIMEOUT = -5
 RR_ERR_TOO_SMALL = -6
+RR_ERR_TOO_LARGE = -7
+RR_NOALLOC_MAX_TILES = 65536
 RR_BF16 = 0
 RR_F32 = 1
 RR_STATUS_TIMEOUT = 1
@@ -82,6 +84,8 @@ def lib() -> C.CDLL:
         L.rr_ledger_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
         L.rr_sampler_draw_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
         L.rr_sampler_draw_u32.restype = C.c_uint32
+        L.rr_compact_flags_noalloc.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+        L.rr_compact_flags_noalloc.restype = C.c_int
         L.rr_profile_begin.argtypes = [vp]
         L.rr_profile_begin.restype = C.c_int
         L.rr_profile_end.argtypes = [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
@@ -181,6 +185,16 @@ def rr_ledger_status(h: int, stream: int) -> int:
 
 def rr_sampler_draw_u32(seed: int, g: int, layer: int, t: int) -> int:
     return int(lib().rr_sampler_draw_u32(seed, g, layer, t))
+
+
+def rr_compact_flags_noalloc(dev_flags: int, n_problems: int, n_q: int, dev_rows_out: int,
+                             dev_count_out: int, dev_problem_offsets_out: int,
+                             stream: int) -> None:
+    """Compaction without any allocation: the scratch is a fixed array inside the library
+    (for callers that may not call cudaMalloc).  Arguments are raw device addresses."""
+    _check(lib().rr_compact_flags_noalloc(dev_flags, n_problems, n_q, dev_rows_out,
+                                          dev_count_out, dev_problem_offsets_out, stream),
+           "rr_compact_flags_noalloc")
 
 
 def rr_profile_begin(h: int) -> None:

@@ -351,6 +351,7 @@ const char* rr_strerror(int code) {
     case RR_ERR_CUDA: return "CUDA runtime error";
     case RR_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case RR_ERR_TOO_SMALL: return "buffer too small";
+    case RR_ERR_TOO_LARGE: return "problem exceeds a fixed built-in capacity";
     default: return "unknown error";
   }
 }
