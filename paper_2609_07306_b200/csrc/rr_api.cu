@@ -113,7 +113,8 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   if (anchor) {
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
     LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, st));
-    LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
+    if (p.dtype == RR_BF16) LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, nullptr, st));
+    else LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
     LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, nullptr, layer, st));
     LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
     L->anchored = 1;
@@ -122,7 +123,10 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
     LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, st));
-    LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
+    if (p.dtype == RR_BF16)
+      LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, p.refresh_rows, st));
+    else
+      LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
     LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, p.refresh_rows, layer, st));
     LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
   }

@@ -80,6 +80,8 @@ __host__ __device__ __forceinline__ uint32_t rr_draw_u32(unsigned long long row_
 // All return cudaError_t from the launch; all are asynchronous on `st`.
 cudaError_t rr_launch_score_simt(const RRParams& p, const void* qc, const void* kc,
                                  const int32_t* row_list, cudaStream_t st);
+cudaError_t rr_launch_score_tc(const RRParams& p, const void* qc, const void* kc,
+                               const int32_t* row_list, cudaStream_t st);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
 cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
