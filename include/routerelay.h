@@ -75,7 +75,9 @@ typedef struct rr_config {
   float   gamma;           /* guard margin of Eq. 5, >= 0 (+inf allowed)                   */
   uint64_t seed;           /* seed of the random-sentinel sampler                          */
   int32_t chunk_tokens;    /* >0: also expand routes to token ranges of this chunk size    */
-  int32_t debug_outputs;   /* 1: relay also stores every candidate score (tests)           */
+  int32_t debug_outputs;   /* bit 0: relay also stores every candidate score (tests);
+                              bit 1: route through the two-pass path (score rows in scratch
+                              + warp-level TopK) even where the fused kernel applies      */
 } rr_config;
 
 /* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */

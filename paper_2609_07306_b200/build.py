@@ -40,7 +40,7 @@ def build(verbose: bool = False, force: bool = False) -> str:
         return LIB
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
            "-std=c++17", "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-           "-o", LIB] + sources()
+           "-o", LIB] + os.environ.get("RR_EXTRA_NVCC_FLAGS", "").split() + sources()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -79,7 +79,7 @@ Layout make_layout(const rr_config* c) {
   L.counters = o;        o = align_up(o + RR_NUM_COUNTERS * 8);
   L.status = o;          o = align_up(o + 4);
   L.token_ranges = o;    o = align_up(o + (c->chunk_tokens > 0 ? rows * c->k * 8 : 0));
-  L.cand_scores = o;     o = align_up(o + (c->debug_outputs ? rows * cw * 4 : 0));
+  L.cand_scores = o;     o = align_up(o + ((c->debug_outputs & 1) ? rows * cw * 4 : 0));
   L.S = o;               o = align_up(o + rows * (size_t)c->n_k * 4);
   L.scratch_total = o;
   return L;
@@ -113,9 +113,13 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   if (anchor) {
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
     LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, st));
-    if (p.dtype == RR_BF16) LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, nullptr, st));
-    else LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
-    LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, nullptr, layer, st));
+    if (L->fused) {
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, nullptr, layer, st));
+    } else {
+      if (p.dtype == RR_BF16) LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, nullptr, st));
+      else LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
+      LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, nullptr, layer, st));
+    }
     LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
     L->anchored = 1;
   } else {
@@ -123,11 +127,15 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
     LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, st));
-    if (p.dtype == RR_BF16)
-      LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, p.refresh_rows, st));
-    else
-      LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
-    LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, p.refresh_rows, layer, st));
+    if (L->fused) {
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
+    } else {
+      if (p.dtype == RR_BF16)
+        LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, p.refresh_rows, st));
+      else
+        LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
+      LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, p.refresh_rows, layer, st));
+    }
     LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
   }
 #undef LAUNCH
@@ -181,7 +189,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.P = cfg->batch * cfg->heads; p.n_q = cfg->n_q; p.n_k = cfg->n_k; p.d = cfg->d;
   p.k = cfg->k; p.m = cfg->m; p.r = cfg->r; p.sw = cfg->m + cfg->r; p.c = cfg->k + p.sw;
   p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
-  p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs;
+  p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs & 1;
   p.rows = p.P * p.n_q;
   p.tiles_per_problem = (p.n_q + RR_ROW_TILE - 1) / RR_ROW_TILE;
   p.n_tiles = p.P * p.tiles_per_problem;
@@ -199,8 +207,9 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.counters = (unsigned long long*)(sb + lay.counters);
   p.status = (uint32_t*)(sb + lay.status);
   p.token_ranges = cfg->chunk_tokens > 0 ? (int32_t*)(sb + lay.token_ranges) : nullptr;
-  p.cand_scores = cfg->debug_outputs ? (float*)(sb + lay.cand_scores) : nullptr;
+  p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
+  L->fused = !(cfg->debug_outputs & 2) && rr_route_fused_supported(p);
   *out = L;
   return RR_OK;
 }

@@ -13,7 +13,7 @@
 // Everything a kernel needs to know about one ledger; passed by value.
 struct RRParams {
   int P, n_q, n_k, d, k, m, r, c, sw;      // sw = m + r (sentinel row width)
-  int dtype, causal, causal_offset, chunk_tokens, debug;
+  int dtype, causal, causal_offset, chunk_tokens, debug;   // debug: bit 0 = store candidate scores
   int rows, tiles_per_problem, n_tiles;    // row tiles of RR_ROW_TILE per problem / in total
   float gamma;
   unsigned long long seed;
@@ -35,6 +35,7 @@ struct rr_ledger {
   size_t export_bytes;
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
+  bool fused;                              // full routing runs in the fused tensor-core kernel
   unsigned long long dense_pairs_per_layer;
   // benchmark-only per-kernel timing
   bool profiling = false;
@@ -82,6 +83,9 @@ cudaError_t rr_launch_score_simt(const RRParams& p, const void* qc, const void* 
                                  const int32_t* row_list, cudaStream_t st);
 cudaError_t rr_launch_score_tc(const RRParams& p, const void* qc, const void* kc,
                                const int32_t* row_list, cudaStream_t st);
+bool rr_route_fused_supported(const RRParams& p);
+cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void* kc,
+                                  const int32_t* row_list, int layer, cudaStream_t st);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
 cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,

@@ -1,0 +1,748 @@
+// Full routing of a set of rows in ONE kernel: score GEMM on the tensor cores (Eq. 1), per-row
+// TopK (Eq. 2), near-miss sentinels (Section 3.1 item 1), k-th score and margin (Section 3.3),
+// random sentinels (Section 3.1 item 2) -- the score matrix never leaves the SM.
+//
+// One CTA owns 128 query rows of one problem (consecutive rows at an anchor; a segment of the
+// compacted refresh list at a relay, Section 4.2) and walks the key chunks in tiles of 64,
+// stopping at the last chunk any of its rows may select.
+//   warp 0   : TMA producer (Kc tiles, 128-byte swizzle, 2-stage ring, no multicast)
+//   warp 1   : one thread issues tcgen05.mma (M=128, N=64, K=16) into a double-buffered TMEM
+//              accumulator
+//   warps 2-5: selection, ONE THREAD PER QUERY ROW (tcgen05.ld 32x32b hands each thread 32
+//              consecutive scores of its own row).  Each thread streams its row through a
+//              threshold filter into a private candidate buffer in shared memory
+//              (order-preserving 32-bit keys + chunk ids, laid out [slot][thread] so that
+//              accesses are bank-conflict free).  When a buffer nears its capacity the warp
+//              re-tightens: a 32-bin histogram over the buffer's key range finds the bin that
+//              holds the KEEP-th largest key (KEEP = k + max(m,1)), the threshold moves to that
+//              bin's lower edge and the buffer is compacted in place (stable, so entries stay
+//              in ascending chunk id).  After the last tile an exact multi-level histogram
+//              select (5 key bits per level) fixes rank KEEP and rank k; ties are resolved
+//              towards the smaller chunk id by buffer order.  The result is exact.
+// Random sentinels are drawn by the same thread with the counter-based generator, using a
+// per-row bitmap of excluded chunks in shared memory.  Every mbarrier wait is bounded.
+#include "rr_common.cuh"
+#include "rr_sm100.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int BM = 128, BN = 64, B_STAGES = 2, ACC_STAGES = 2, NT = 192;
+constexpr int TMEM_COLS = ACC_STAGES * BN;
+constexpr int NB = 32, NB_LOG = 5;             // histogram bins per level
+constexpr int CHUNK = 32;                      // scores handed to a thread per TMEM load
+constexpr unsigned FULL = 0xFFFFFFFFu;
+
+template <int D>
+struct Cfg {
+  static constexpr int KHALVES = D / 64, KSTEPS = D / 16;
+  static constexpr int A_BYTES = BM * D * 2, B_BYTES = BN * D * 2;
+  static constexpr int A_HALF = BM * 128, B_HALF = BN * 128;   // rows x 128 bytes (64 bf16)
+  static constexpr int CTL_BYTES = 2048;
+  static constexpr int FIXED_BYTES = 1024 + A_BYTES + B_STAGES * B_BYTES + CTL_BYTES;
+};
+
+struct Ctl {
+  uint64_t full[B_STAGES], empty[B_STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+  uint32_t tmem_base, abort_flag;
+  int row[BM], slot[BM];
+};
+
+// ---- thread-private selection state ---------------------------------------------------------
+// A row's candidate buffer holds 8-byte entries {score bits, chunk id}; entry e of the thread
+// that owns row r lives at buf + e*ENTRY_PITCH (ENTRY_PITCH = 128 rows * 8 bytes), so a warp's
+// accesses to "entry e_lane" are bank-conflict free whatever e_lane is.  Histogram bins and
+// the exclusion bitmap are 32-bit words at aux + b*AUX_PITCH.  All accesses use explicit
+// shared-window addresses (32-bit) and ld/st/red.shared.
+constexpr uint32_t ENTRY_PITCH = BM * 8, AUX_PITCH = BM * 4;
+struct Sel { uint32_t buf, aux; };
+
+__device__ __forceinline__ void st_entry(uint32_t addr, float s, uint32_t id) {
+  asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "f"(s), "r"(id) : "memory");
+}
+__device__ __forceinline__ void ld_entry(uint32_t addr, float& s, uint32_t& id) {
+  asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=f"(s), "=r"(id) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ float ld_score(uint32_t addr) {
+  float s;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=f"(s) : "r"(addr) : "memory");
+  return s;
+}
+__device__ __forceinline__ uint32_t aux_ld(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void aux_st(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void aux_inc(uint32_t addr) {
+  asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+// predicated forms: no branch is emitted, the access is simply masked off
+__device__ __forceinline__ void st_entry_if(bool pred, uint32_t addr, float s, uint32_t id) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.shared.v2.b32 [%0], {%1, %2};\n\t}"
+               ::"r"(addr), "f"(s), "r"(id), "r"((uint32_t)pred) : "memory");
+}
+__device__ __forceinline__ void aux_inc_if(bool pred, uint32_t addr) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p red.shared.add.u32 [%0], 1;\n\t}"
+               ::"r"(addr), "r"((uint32_t)pred) : "memory");
+}
+__device__ __forceinline__ void aux_or(uint32_t addr, uint32_t bits) {
+  asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(bits) : "memory");
+}
+
+// All passes over a buffer walk it in batches of 8 with the loads issued first: a thread's
+// passes are chains of shared-memory accesses, and with one selection warp per scheduler
+// nothing else hides that latency.  Histogram increments are fire-and-forget reductions.
+//
+// Control flow is kept WARP-UNIFORM: every routine below is called by all 32 lanes, loops run
+// to the warp-wide maximum trip count and each lane masks its own tail, and data-dependent
+// decisions (another refinement level, the key-space fallback) are taken by warp vote.  Lanes
+// that have nothing to do pass n = 0.  Divergent versions of the same passes executed each
+// pass once per divergent lane group and were several times slower.
+constexpr int BATCH = 8;
+
+// Optional phase timing (compile with -DRR_PHASE_TIMING): cycles and event counts per phase,
+// summed over selection warps (lane 0), read back with rr_debug_phase_counters().
+#ifdef RR_PHASE_TIMING
+__device__ unsigned long long g_phase[16];
+#define PH_T0() const long long ph_t0_ = clock64()
+#define PH_ADD(i) do { if ((threadIdx.x & 31) == 0) atomicAdd(&g_phase[i], (unsigned long long)(clock64() - ph_t0_)); } while (0)
+#define PH_CNT(i, val_) do { if ((threadIdx.x & 31) == 0) atomicAdd(&g_phase[i], (unsigned long long)(val_)); } while (0)
+#else
+#define PH_T0() do {} while (0)
+#define PH_ADD(i) do {} while (0)
+#define PH_CNT(i, val_) do {} while (0)
+#endif
+
+__device__ __forceinline__ int warp_max(int x) { return __reduce_max_sync(FULL, x); }
+
+// order-preserving key of a canonical (no -0.0) score
+__device__ __forceinline__ uint32_t key_of(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Finds, in the histogram the lane just built, the bin that holds its need-th largest entry.
+__device__ __forceinline__ void scan_bins(const Sel& s, int need, int& bsel, int& cnt, int& above) {
+  uint32_t h[NB];
+#pragma unroll
+  for (int b = 0; b < NB; ++b) h[b] = aux_ld(s.aux + b * AUX_PITCH);
+  int cum = 0; bsel = 0; cnt = 0; above = 0; bool found = false;
+#pragma unroll
+  for (int b = NB - 1; b >= 0; --b) {
+    const int c = (int)h[b];
+    if (!found && cum + c >= need) { bsel = b; cnt = c; above = cum; found = true; }
+    cum += c;
+  }
+}
+__device__ __forceinline__ void clear_bins(const Sel& s) {
+#pragma unroll
+  for (int b = 0; b < NB; ++b) aux_st(s.aux + b * AUX_PITCH, 0u);
+}
+// Lanes that only tag along in a warp-uniform routine must keep their persistent bins.
+__device__ __forceinline__ void clear_bins_if(bool pred, const Sel& s) {
+  if (pred) clear_bins(s);
+}
+
+// One refinement level in the SCORE domain over the lane's entries with lo <= score <= hi:
+// NB equal-width bins (bin = floor((score - lo) * scale), monotone in the score; equal-width
+// bins of the 32-bit keys would be useless across a sign change or several binades).  Finds
+// the bin b* holding the rank-th largest in-range entry, the number of in-range entries above
+// b* and the score bounds [blo, bhi] of the entries in b*.  With `drop`, entries below b* (and
+// below lo) are removed, stably and in place, and n is updated.
+// Returns false, changing nothing, for lanes with n = 0 or an unusable range.
+__device__ __forceinline__ bool lin_level(const Sel& s, int& n, int nw, float lo, float hi, int rank,
+                                          bool drop, int& cnt, int& above, float& blo, float& bhi) {
+  const float scale = (float)NB / (hi - lo);
+  const bool valid = n > 0 && hi > lo && scale < 1e37f;
+  const int ne = valid ? n : 0;
+  PH_CNT(12, 1); PH_CNT(7, nw);
+  clear_bins_if(valid, s);
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(ne - 1, 0)) * ENTRY_PITCH);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      // plain read-modify-write: the bins are private to this thread, and shared-memory
+      // reductions measured several times slower than a load/add/store chain here
+      const bool in = (e0 + j < ne) & (v[j] >= lo) & (v[j] <= hi);
+      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - lo) * scale)));
+      const uint32_t a = s.aux + b * AUX_PITCH;
+      aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+    }
+  }
+  int bsel;
+  scan_bins(s, rank, bsel, cnt, above);
+  blo = __int_as_float(0x7f800000); bhi = __int_as_float(0xff800000);
+  uint32_t waddr = s.buf;
+  const int ne_last = max(ne - 1, 0);
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH]; uint32_t id[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)      // reading past the lane's count is harmless (< cap)
+      ld_entry(s.buf + min(e0 + j, ne_last) * ENTRY_PITCH, v[j], id[j]);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const bool live = e0 + j < ne;
+      const bool in = live & (v[j] >= lo) & (v[j] <= hi);
+      const int b = min(NB - 1, __float2int_rz((v[j] - lo) * scale));
+      const bool tgt = in & (b == bsel);
+      blo = fminf(blo, tgt ? v[j] : blo); bhi = fmaxf(bhi, tgt ? v[j] : bhi);
+      const bool keep = drop & live & ((v[j] > hi) | (in & (b >= bsel)));
+      st_entry_if(keep, waddr, v[j], id[j]);
+      waddr += keep ? ENTRY_PITCH : 0u;
+    }
+  }
+  if (valid && drop) n = (int)((waddr - s.buf) / ENTRY_PITCH);
+  return valid;
+}
+
+// Key-space fallback (5 key bits per level) for ranges the score-domain levels cannot split
+// (differences too small to scale).  Exact key of rank T among the entries whose keys lie in
+// [lo, hi]; `need` of the entries equal to it belong to the top T.
+__device__ void select_keys(const Sel& s, int n, int T, uint32_t lo, uint32_t hi, uint32_t& key_T,
+                            int& need_out) {
+  const int nw = warp_max(n);
+  uint32_t span = n > 0 ? hi - lo : 0u;
+  int need = T;
+  for (int level = 0; level < 8; ++level) {
+    const bool work = n > 0 && span != 0;
+    if (!__any_sync(FULL, work)) break;
+    const int ne = work ? n : 0;
+    const int shift = max(0, (32 - __clz(span | 1u)) - NB_LOG);
+    clear_bins_if(work, s);
+    for (int e0 = 0; e0 < nw; e0 += BATCH) {
+      float v[BATCH];
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) v[j] = e0 + j < ne ? ld_score(s.buf + (e0 + j) * ENTRY_PITCH) : 0.f;
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) {
+        const uint32_t off = key_of(v[j]) - lo;
+        if (e0 + j < ne && off <= span) aux_inc(s.aux + (off >> shift) * AUX_PITCH);
+      }
+    }
+    int bsel, cnt, above;
+    scan_bins(s, need, bsel, cnt, above);
+    if (work) {
+      need -= above;
+      const uint32_t base = (uint32_t)bsel << shift;
+      lo += base;
+      span = min(span - base, (shift ? (1u << shift) : 1u) - 1u);
+    }
+  }
+  key_T = lo; need_out = need;
+}
+
+// Exact score of rank T (1-based, descending) among the n entries of each participating lane
+// (T <= n; other lanes pass active = false), by zooming score-domain levels until the bin
+// holding rank T contains equal scores only.  `need` of the entries equal to the result belong
+// to the top T.  With `drop`, entries known to rank below T are removed on the way.
+// With fit_limit >= 0 a lane stops as soon as its buffer has shrunk to fit_limit or fewer
+// entries; it then reports exact = false and s_T = the smallest surviving score.
+__device__ void select_rank(const Sel& s, bool active, int& n, int T, bool drop, int fit_limit,
+                            float lo, float hi, float& s_T, int& need, bool& exact) {
+  bool done = !active, fallback = false;
+  int rank = T;
+  exact = false; need = 0; s_T = lo;
+  for (int level = 0; level < 10; ++level) {
+    const bool work = !done;
+    if (!__any_sync(FULL, work)) break;
+    int nl = work ? n : 0;
+    const int n_before = nl;
+    const int nw = warp_max(nl);
+    int cnt, above; float blo, bhi;
+    const bool valid = lin_level(s, nl, nw, lo, hi, rank, drop, cnt, above, blo, bhi);
+    if (work) {
+      if (!valid) { fallback = true; done = true; }
+      else {
+        n = nl;
+        rank -= above;
+        if (blo == bhi) { s_T = blo; need = rank; exact = true; done = true; }
+        else if (fit_limit >= 0 && n <= fit_limit && n < n_before) { s_T = blo; done = true; }
+        else {
+          // zoom into [blo, bhi]; with drop the entries above stay in the buffer, so the
+          // rank inside the bin is what remains to be resolved
+          lo = blo; hi = bhi;
+        }
+      }
+    }
+  }
+  fallback = fallback || !done;
+  if (__any_sync(FULL, fallback)) {
+    PH_CNT(9, 1);
+    uint32_t kt = 0; int nd = 0;
+    select_keys(s, fallback ? n : 0, rank, key_of(lo), key_of(hi), kt, nd);
+    if (fallback) { s_T = rr_key_to_float(kt); need = nd; exact = true; }
+  }
+}
+
+// Keeps scores > s_T and the first `need` entries equal to it (stable, in place).
+__device__ __forceinline__ int compact_exact(const Sel& s, int n, float s_T, int need) {
+  const int nw = warp_max(n);
+  uint32_t waddr = s.buf;
+  int ties = 0;
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH]; uint32_t id[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)
+      ld_entry(s.buf + min(e0 + j, max(n - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const bool in = e0 + j < n;
+      const bool eq = in & (v[j] == s_T);
+      const bool keep = in & ((v[j] > s_T) | (eq & (ties < need)));
+      ties += eq;
+      st_entry_if(keep, waddr, v[j], id[j]);
+      waddr += keep ? ENTRY_PITCH : 0u;
+    }
+  }
+  return (int)((waddr - s.buf) / ENTRY_PITCH);
+}
+
+// Per-row state of the streaming threshold filter.
+struct RowState {
+  float tau;          // pass threshold of the filter (inclusive)
+  float blo;          // lower bound of the buffered scores
+  float smin, smax;   // bounds of all valid scores seen
+  float map_lo, map_scale;   // fixed score -> bin map of the persistent histogram
+  int binned;         // buffer entries [0, binned) are counted in the histogram; -1: no map yet
+};
+
+// Re-tightening with a PERSISTENT histogram: the row's score->bin map is fixed at its first
+// re-tightening (NB equal bins over the range seen so far; later, larger scores fall into the
+// top bin), so each call only has to bin the entries appended since the previous call, find
+// the bin b* of rank `keep` from the top, and drop the entries below b* (stable, in place).
+// Bins below b* keep stale counts, which is harmless: the threshold only rises.  If b* is too
+// crowded for the buffer to fit `fit_limit`, score-domain zoom levels finish the job and the
+// histogram is rebuilt at the next call.
+// fit_limit < 0 asks for the exact cut at rank `keep` (n becomes exactly keep).
+__device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_limit, RowState& st) {
+  // (1) map + binning of the new entries
+  const bool fresh = active && st.binned < 0;
+  if (fresh) {
+    st.map_lo = st.smin;
+    st.map_scale = (float)NB / (st.smax - st.smin);
+    st.binned = 0;
+  }
+  const bool usable = active && st.smax > st.smin && st.map_scale < 1e37f;
+  if (__any_sync(FULL, fresh)) {
+    if (fresh) clear_bins(s);
+  }
+  const int from = usable ? st.binned : 0, to = usable ? n : 0;
+  const int nw_new = warp_max(to - from);
+  const float mlo = st.map_lo, msc = st.map_scale;
+  for (int e0 = 0; e0 < nw_new; e0 += BATCH) {
+    float v[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)
+      v[j] = ld_score(s.buf + min(from + e0 + j, max(to - 1, 0)) * ENTRY_PITCH);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const bool in = from + e0 + j < to;
+      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+      const uint32_t a = s.aux + b * AUX_PITCH;
+      aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+    }
+  }
+  // (2) bin of rank keep, drop what lies below it
+  int bsel, cnt, above;
+  scan_bins(s, keep, bsel, cnt, above);
+  const int nd = usable ? n : 0;
+  const int nw = warp_max(nd);
+  uint32_t waddr = s.buf;
+  float blo = __int_as_float(0x7f800000), bhi = __int_as_float(0xff800000);   // bounds of bin b*
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH]; uint32_t id[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)
+      ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+      const bool live = e0 + j < nd;
+      const bool keep_it = live & (b >= bsel), tgt = live & (b == bsel);
+      blo = fminf(blo, tgt ? v[j] : blo); bhi = fmaxf(bhi, tgt ? v[j] : bhi);
+      st_entry_if(keep_it, waddr, v[j], id[j]);
+      waddr += keep_it ? ENTRY_PITCH : 0u;
+    }
+  }
+  if (usable) {
+    n = (int)((waddr - s.buf) / ENTRY_PITCH);
+    st.binned = n;
+    st.blo = blo; st.tau = blo;       // >= keep seen scores reach blo: a valid threshold
+  }
+  // (3) crowded bin or unusable range: zoom levels / exact cut
+  const bool more = active && (!usable || n > fit_limit);
+  if (__any_sync(FULL, more)) {
+    PH_CNT(9, 1);
+    float s_T; int need; bool exact;
+    // usable: everything left of interest is inside bin b* = [blo, bhi], `above` entries
+    // outrank it; otherwise the whole buffer is searched
+    select_rank(s, more, n, usable ? keep - above : keep, true, fit_limit,
+                usable ? blo : fminf(st.blo, st.smin), usable ? bhi : st.smax, s_T, need, exact);
+    const int w = compact_exact(s, more && exact ? n : 0, s_T, need);
+    if (more) {
+      if (exact) { n = w; st.tau = rr_key_to_float(key_of(s_T) + 1u); }   // later ties lose
+      else st.tau = s_T;
+      st.blo = s_T;
+      // the scratch levels overwrote the bins: rebuild from the buffer at the next call
+      st.binned = usable ? 0 : -1;       // unusable range: choose a new map next time
+      clear_bins(s);
+    }
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(NT, 1)
+route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
+                   const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
+                   uint32_t layer, int cap, int aux_words) {
+  using C = Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + C::A_BYTES;
+  Ctl* ctl = (Ctl*)(smem + C::A_BYTES + B_STAGES * C::B_BYTES);
+  uint8_t* s_buf = (uint8_t*)ctl + C::CTL_BYTES;                      // [cap][BM] 8-byte entries
+  uint8_t* s_aux = s_buf + (size_t)cap * ENTRY_PITCH;                 // [aux_words][BM] words
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tiles_m = p.tiles_per_problem;
+  const int prob = blockIdx.x / tiles_m, tm = blockIdx.x % tiles_m;
+
+  int seg_lo = 0, seg_hi = p.n_q;
+  if (row_list) { seg_lo = p.problem_offsets[prob]; seg_hi = p.problem_offsets[prob + 1]; }
+  if (tm * BM >= seg_hi - seg_lo) return;                 // nothing to do (uniform per CTA)
+
+  if (tid < BM) {
+    const int local = tm * BM + tid;
+    int row = -1, slot = 0;
+    if (row_list) {
+      const int s = seg_lo + local;
+      if (s < seg_hi) { row = row_list[s] - prob * p.n_q; slot = s; }
+    } else if (local < p.n_q) {
+      row = local; slot = prob * p.n_q + local;
+    }
+    ctl->row[tid] = row; ctl->slot[tid] = slot;
+  }
+  if (tid == 0) {
+    for (int s = 0; s < B_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(&ctl->acc_full[s], 1); mbar_init(&ctl->acc_empty[s], BM); }
+    ctl->abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmap_k);
+  }
+  if (warp == 0) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+  __syncthreads();
+
+  // ---- gather the Qc tile into the K-major, 128B-swizzled layout -------------------------
+  {
+    constexpr int CPR = D / 8;
+    const __nv_bfloat16* qbase = qc + (size_t)prob * p.n_q * D;
+    for (int ch = tid; ch < BM * CPR; ch += NT) {
+      const int r = ch / CPR, c16 = ch % CPR, h = c16 >> 3, cc = c16 & 7;
+      const int row = ctl->row[r];
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (row >= 0) v = __ldg(reinterpret_cast<const uint4*>(qbase + (size_t)row * D + c16 * 8));
+      *reinterpret_cast<uint4*>(sA + h * C::A_HALF + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+  int last = -1;
+  for (int t = BM - 1; t >= 0; --t) if (ctl->row[t] >= 0) { last = ctl->row[t]; break; }
+  const int vmax = rr_valid_count(last, p.n_k, p.causal, p.causal_offset);
+  const int n_tiles = (vmax + BN - 1) / BN;
+
+  if (warp == 0) {
+    // ===== TMA producer =====
+    if (lane == 0) {
+      int issued = 0;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
+        if (!mbar_wait(&ctl->empty[s], ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(&ctl->full[s], C::B_BYTES);
+#pragma unroll
+        for (int h = 0; h < C::KHALVES; ++h)
+          tma_load_3d(sB + s * C::B_BYTES + h * C::B_HALF, &tmap_k, h * 64, t * BN, prob,
+                      &ctl->full[s]);
+        ++issued;
+      }
+      for (int t = max(0, issued - B_STAGES); t < issued; ++t) {
+        const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->full[s], ph); ++it) __nanosleep(64);
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer =====
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+      const uint32_t a_addr = smem_u32(sA);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
+        const int as = t % ACC_STAGES; const uint32_t aph = (t / ACC_STAGES) & 1;
+        if (!mbar_wait(&ctl->acc_empty[as], aph ^ 1, abort_flag)) break;
+        if (!mbar_wait(&ctl->full[s], ph, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t b_addr = smem_u32(sB + s * C::B_BYTES);
+#pragma unroll
+        for (int k = 0; k < C::KSTEPS; ++k) {
+          const uint32_t a_off = (k >> 2) * C::A_HALF + (k & 3) * 32;
+          const uint32_t b_off = (k >> 2) * C::B_HALF + (k & 3) * 32;
+          umma_bf16(tmem_base + as * BN, umma_desc_k_sw128(a_addr + a_off),
+                    umma_desc_k_sw128(b_addr + b_off), idesc, k > 0 ? 1u : 0u);
+        }
+        umma_commit(&ctl->empty[s]);
+        umma_commit(&ctl->acc_full[as]);
+      }
+    }
+  } else {
+    // ===== selection: one thread per query row =====
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;
+    const int row = ctl->row[r];
+    const int v = row >= 0 ? rr_valid_count(row, p.n_k, p.causal, p.causal_offset) : 0;
+    const int keep_cfg = p.k + max(p.m, 1);
+    const int keep = min(keep_cfg, v), kk = min(p.k, v);
+    const Sel sel{smem_u32(s_buf) + r * 8u, smem_u32(s_aux) + r * 4u};
+    const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
+    RowState st;
+    st.tau = row >= 0 ? ninf : pinf;          // padding rows pass nothing
+    st.blo = pinf; st.smin = pinf; st.smax = ninf;
+    st.map_lo = 0.f; st.map_scale = 0.f; st.binned = -1;
+    uint32_t waddr = sel.buf;                 // next free entry
+    const uint32_t trigger = sel.buf + (uint32_t)(cap - CHUNK) * ENTRY_PITCH;
+    int vmaxw = v, vminw = row >= 0 ? v : 0x7FFFFFFF;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+      vmaxw = max(vmaxw, __shfl_xor_sync(FULL, vmaxw, off));
+      vminw = min(vminw, __shfl_xor_sync(FULL, vminw, off));
+    }
+    bool alive = true;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int as = t % ACC_STAGES; const uint32_t aph = (t / ACC_STAGES) & 1;
+      bool ready;
+      { PH_T0(); ready = mbar_wait(&ctl->acc_full[as], aph, abort_flag); PH_ADD(0); }
+      if (!__all_sync(FULL, ready)) { alive = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < BN / CHUNK; ++c) {
+        const int col0 = t * BN + c * CHUNK;
+        if (col0 >= vmaxw) break;                          // no row of this warp sees these
+        if (__any_sync(FULL, waddr > trigger)) {
+          // re-tighten: raise the threshold until the buffer fits again
+          PH_T0();
+          int n = (int)((waddr - sel.buf) / ENTRY_PITCH);
+          const bool act = n > keep;
+          retighten(sel, act, n, keep, (keep + cap - CHUNK) / 2, st);
+          if (act) waddr = sel.buf + (uint32_t)n * ENTRY_PITCH;
+          PH_ADD(1); PH_CNT(8, 1);
+        }
+        PH_T0();
+        const float tau_f = st.tau;
+        uint32_t acc[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + c * CHUNK, acc);
+        // threshold filter: branch-free appends (predicated stores); waddr is the only chain
+        if (col0 + CHUNK <= vminw) {
+#pragma unroll
+          for (int q = 0; q < CHUNK; ++q) {
+            const float sc = __uint_as_float(acc[q]) + 0.0f;         // -0.0 -> +0.0
+            const bool pass = sc >= tau_f;
+            st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc);
+            if (pass) st_entry(waddr, sc, (uint32_t)(col0 + q));
+            waddr += pass ? ENTRY_PITCH : 0u;
+          }
+        } else {
+#pragma unroll
+          for (int q = 0; q < CHUNK; ++q) {
+            const float sc = __uint_as_float(acc[q]) + 0.0f;
+            const bool valid = col0 + q < v;
+            const bool pass = valid && sc >= tau_f;
+            if (valid) { st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc); }
+            if (pass) st_entry(waddr, sc, (uint32_t)(col0 + q));
+            waddr += pass ? ENTRY_PITCH : 0u;
+          }
+        }
+        PH_ADD(2); PH_CNT(10, 1);
+      }
+      tc_fence_before();
+      mbar_arrive(&ctl->acc_empty[as]);
+    }
+
+    if (alive) {                                    // warp-uniform
+      const bool have = row >= 0;
+      const int g = have ? (row_list ? row_list[ctl->slot[r]] : ctl->slot[r]) : 0;
+      int n = have ? (int)((waddr - sel.buf) / ENTRY_PITCH) : 0;
+      PH_CNT(11, 1);
+      // ---- exact cut at rank keep ---------------------------------------------------------------
+      {
+        PH_T0();
+        const bool cut = n > keep;
+        retighten(sel, cut, n, keep, -1, st);
+        PH_ADD(3);
+      }
+      // ---- split at rank kk ---------------------------------------------------------------------
+      float s_k = ninf; int need_k = 0;
+      {
+        PH_T0();
+        const bool split = n > kk;
+        int n_ = n; bool exact;
+        select_rank(sel, split, n_, kk, false, -1, fminf(st.blo, st.smin), st.smax, s_k, need_k, exact);
+        if (!split) { s_k = ninf; need_k = 0; }       // everything buffered is selected
+        PH_ADD(4);
+      }
+      PH_T0();
+      for (int w = 0; w < aux_words; ++w) aux_st(sel.aux + w * AUX_PITCH, 0u);   // exclusion bitmap
+      int32_t* route = p.routes + (size_t)g * p.k;
+      int32_t* sent = p.sentinels + (size_t)g * p.sw;
+      int nr = 0, nn = 0, ties = 0, cur_word = -1;
+      uint32_t cur_bits = 0u;
+      float kth = pinf, next = ninf;
+      const int nw = warp_max(n);
+      for (int e0 = 0; e0 < nw; e0 += BATCH) {
+        float sv[BATCH]; uint32_t id[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+          sv[j] = 0.f; id[j] = 0;
+          if (e0 + j < n) ld_entry(sel.buf + (e0 + j) * ENTRY_PITCH, sv[j], id[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+          if (e0 + j < n) {
+            const bool eq = sv[j] == s_k;
+            const bool in_route = sv[j] > s_k || (eq && ties < need_k);
+            ties += eq;
+            bool excluded = in_route;
+            if (in_route) {
+              route[nr++] = (int)id[j]; kth = fminf(kth, sv[j]);
+            } else {
+              next = fmaxf(next, sv[j]);
+              if (nn < p.m) { sent[nn++] = (int)id[j]; excluded = true; }
+            }
+            // entries are in ascending chunk id: a bitmap word is complete when the id moves
+            // past it, so it is written once, with no read-modify-write
+            const int wi = (int)(id[j] >> 5);
+            if (wi != cur_word) {
+              if (cur_word >= 0) aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
+              cur_word = wi; cur_bits = 0u;
+            }
+            cur_bits |= excluded ? 1u << (id[j] & 31) : 0u;
+          }
+        }
+      }
+      if (cur_word >= 0) aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
+      PH_ADD(5);
+      if (have) {
+        PH_T0();
+        for (int e = nr; e < p.k; ++e) route[e] = -1;
+        for (int e = nn; e < p.m; ++e) sent[e] = -1;
+        p.kth[g] = kth;
+        p.margin[g] = v > kk ? kth - next : pinf;
+
+        // ---- random sentinels --------------------------------------------------------------
+        int32_t* rnd = sent + p.m;
+        const int pool = v - (nr + nn);
+        int taken = 0;
+        if (p.r > 0 && pool > 0) {
+          if (pool > p.r) {
+            const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
+            const int limit = 64 * p.r;
+            for (int t = 0; t < limit && taken < p.r; ++t) {
+              const int j = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)t), (uint32_t)v);
+              const uint32_t wa = sel.aux + (j >> 5) * AUX_PITCH;
+              const uint32_t w = aux_ld(wa), bit = 1u << (j & 31);
+              if (!(w & bit)) { aux_st(wa, w | bit); rnd[taken++] = j; }
+            }
+          }
+          for (int j = 0; j < v && taken < p.r; ++j)
+            if (!((aux_ld(sel.aux + (j >> 5) * AUX_PITCH) >> (j & 31)) & 1u)) rnd[taken++] = j;
+        }
+        for (int e = taken; e < p.r; ++e) rnd[e] = -1;
+        PH_ADD(6);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+    if (lane == 0 && ctl->abort_flag) atomicOr(p.status, RR_STATUS_TIMEOUT);
+  }
+}
+
+// Shared-memory plan: returns false if the configuration does not fit the fused kernel.
+bool plan(const RRParams& p, int& cap, int& aux_words, size_t& smem_bytes) {
+  const int keep = p.k + (p.m > 0 ? p.m : 1);
+  const size_t fixed = p.d == 128 ? Cfg<128>::FIXED_BYTES : Cfg<64>::FIXED_BYTES;
+  aux_words = (p.n_k + 31) / 32;
+  if (aux_words < NB) aux_words = NB;
+  const size_t max_smem = 227 * 1024;
+  const size_t aux = (size_t)aux_words * BM * 4;
+  if (fixed + aux >= max_smem) return false;
+  const size_t per_entry = ENTRY_PITCH;
+  int fit = (int)((max_smem - fixed - aux) / per_entry);
+  cap = keep + 96;
+  if (cap > fit) cap = fit;
+  if (cap < keep + CHUNK) return false;
+  if (p.n_k > 65535) return false;
+  smem_bytes = fixed + aux + (size_t)cap * per_entry;
+  return true;
+}
+
+}  // namespace
+
+#ifdef RR_PHASE_TIMING
+extern "C" int rr_debug_phase_counters(unsigned long long* out16, int reset) {
+  cudaDeviceSynchronize();
+  if (cudaMemcpyFromSymbol(out16, g_phase, sizeof(unsigned long long) * 16) != cudaSuccess) return -1;
+  if (reset) {
+    unsigned long long z[16] = {};
+    cudaMemcpyToSymbol(g_phase, z, sizeof z);
+  }
+  return 0;
+}
+#endif
+
+bool rr_route_fused_supported(const RRParams& p) {
+  int cap, aux; size_t smem;
+  return p.dtype == RR_BF16 && plan(p, cap, aux, smem);
+}
+
+cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void* kc,
+                                  const int32_t* row_list, int layer, cudaStream_t st) {
+  int cap, aux; size_t smem;
+  if (!plan(p, cap, aux, smem)) return cudaErrorInvalidConfiguration;
+  CUtensorMap tmap;
+  cudaError_t e = rr_encode_tmap_bf16_3d(&tmap, kc, p.d, p.n_k, p.P, BN);
+  if (e != cudaSuccess) return e;
+  const int grid = p.P * p.tiles_per_problem;
+  static bool attr_set = false;
+  if (!attr_set) {
+    e = cudaFuncSetAttribute(route_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(route_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  if (p.d == 128)
+    route_fused_kernel<128><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, row_list,
+                                                    (uint32_t)layer, cap, aux);
+  else
+    route_fused_kernel<64><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, row_list,
+                                                   (uint32_t)layer, cap, aux);
+  rr_count_launch();
+  return cudaPeekAtLastError();
+}

@@ -25,16 +25,18 @@ def test_tiny_fp32_all_layers():
     parity.assert_clean(rep)
 
 
-def test_moderate_bf16_causal_all_layers():
-    rep = parity.run_teacher_forced(W.moderate())
+@pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
+def test_moderate_bf16_causal_all_layers(two_pass):
+    rep = parity.run_teacher_forced(W.moderate(), two_pass=two_pass)
     _report(rep)
     parity.assert_clean(rep)
 
 
+@pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
 @pytest.mark.parametrize("n", [128, 512])
-def test_sweep_shapes(n):
+def test_sweep_shapes(n, two_pass):
     w = W.sweep(n, 0.15).replace(heads=4, layers=4, anchor_every=3)
-    rep = parity.run_teacher_forced(w)
+    rep = parity.run_teacher_forced(w, two_pass=two_pass)
     _report(rep)
     parity.assert_clean(rep)
 
@@ -43,9 +45,10 @@ def test_ragged_shapes_and_wide_ledger():
     # n_q not a multiple of any tile, n_q != n_k, non-causal, d=64 bf16, wide candidate set
     w = W.RouteWorkload("ragged", 1, 3, 200, 333, 64, 12, 24, 12, layers=3, anchor_every=3,
                         dtype=W.DTYPE_BF16, centroids=16, rho=0.05, causal=False, seed=3)
-    rep = parity.run_teacher_forced(w)
-    _report(rep)
-    parity.assert_clean(rep)
+    for two_pass in (False, True):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass)
+        _report(rep)
+        parity.assert_clean(rep)
     w = W.RouteWorkload("ragged32", 2, 1, 130, 130, 128, 5, 0, 7, layers=3, anchor_every=2,
                         dtype=W.DTYPE_F32, centroids=8, rho=0.1, causal=True, seed=4)
     rep = parity.run_teacher_forced(w)
