@@ -28,7 +28,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int BM = 128, BN = 64, B_STAGES = 2, ACC_STAGES = 2, NT = 192;
+constexpr int BM = 128, BN = 64, B_STAGES = 2, ACC_STAGES = 4, NT = 192;
 constexpr int TMEM_COLS = ACC_STAGES * BN;
 constexpr int NB = 32, NB_LOG = 5;             // histogram bins per level
 constexpr int CHUNK = 32;                      // scores handed to a thread per TMEM load
@@ -147,6 +147,33 @@ __device__ __forceinline__ void clear_bins_if(bool pred, const Sel& s) {
   if (pred) clear_bins(s);
 }
 
+// What a narrowing pass learns about the bin that holds the wanted rank: how many entries it
+// has, how many in-range entries outrank it, and its two largest / two smallest scores --
+// enough to finish exactly, without another level, whenever the bin has at most 4 entries.
+struct BinInfo {
+  int cnt, above;
+  float mx1, mx2, mn2, mn1;          // mx1 >= mx2 >= ... >= mn2 >= mn1 (bin bounds: mn1, mx1)
+  __device__ __forceinline__ void reset() {
+    mx1 = mx2 = __int_as_float(0xff800000); mn1 = mn2 = __int_as_float(0x7f800000);
+  }
+  __device__ __forceinline__ void track(bool tgt, float v) {
+    const float vm = tgt ? v : __int_as_float(0xff800000);
+    mx2 = fmaxf(mx2, fminf(mx1, vm)); mx1 = fmaxf(mx1, vm);
+    const float vn = tgt ? v : __int_as_float(0x7f800000);
+    mn2 = fminf(mn2, fmaxf(mn1, vn)); mn1 = fminf(mn1, vn);
+  }
+  // rank r (1-based from the top) inside the bin, cnt <= 4 or all entries equal.
+  __device__ __forceinline__ bool resolve(int r, float& s_T, int& need) const {
+    if (mx1 == mn1) { s_T = mx1; need = r; return true; }
+    if (cnt > 4) return false;
+    const float l0 = mx1, l1 = cnt == 2 ? mn1 : mx2, l2 = cnt == 3 ? mn1 : mn2, l3 = mn1;
+    s_T = r == 1 ? l0 : r == 2 ? l1 : r == 3 ? l2 : l3;
+    const int g = (l0 > s_T) + (cnt > 1 && l1 > s_T) + (cnt > 2 && l2 > s_T) + (cnt > 3 && l3 > s_T);
+    need = r - g;
+    return true;
+  }
+};
+
 // One refinement level in the SCORE domain over the lane's entries with lo <= score <= hi:
 // NB equal-width bins (bin = floor((score - lo) * scale), monotone in the score; equal-width
 // bins of the 32-bit keys would be useless across a sign change or several binades).  Finds
@@ -155,7 +182,7 @@ __device__ __forceinline__ void clear_bins_if(bool pred, const Sel& s) {
 // below lo) are removed, stably and in place, and n is updated.
 // Returns false, changing nothing, for lanes with n = 0 or an unusable range.
 __device__ __forceinline__ bool lin_level(const Sel& s, int& n, int nw, float lo, float hi, int rank,
-                                          bool drop, int& cnt, int& above, float& blo, float& bhi) {
+                                          bool drop, BinInfo& bi) {
   const float scale = (float)NB / (hi - lo);
   const bool valid = n > 0 && hi > lo && scale < 1e37f;
   const int ne = valid ? n : 0;
@@ -176,8 +203,8 @@ __device__ __forceinline__ bool lin_level(const Sel& s, int& n, int nw, float lo
     }
   }
   int bsel;
-  scan_bins(s, rank, bsel, cnt, above);
-  blo = __int_as_float(0x7f800000); bhi = __int_as_float(0xff800000);
+  scan_bins(s, rank, bsel, bi.cnt, bi.above);
+  bi.reset();
   uint32_t waddr = s.buf;
   const int ne_last = max(ne - 1, 0);
   for (int e0 = 0; e0 < nw; e0 += BATCH) {
@@ -190,8 +217,7 @@ __device__ __forceinline__ bool lin_level(const Sel& s, int& n, int nw, float lo
       const bool live = e0 + j < ne;
       const bool in = live & (v[j] >= lo) & (v[j] <= hi);
       const int b = min(NB - 1, __float2int_rz((v[j] - lo) * scale));
-      const bool tgt = in & (b == bsel);
-      blo = fminf(blo, tgt ? v[j] : blo); bhi = fmaxf(bhi, tgt ? v[j] : bhi);
+      bi.track(in & (b == bsel), v[j]);
       const bool keep = drop & live & ((v[j] > hi) | (in & (b >= bsel)));
       st_entry_if(keep, waddr, v[j], id[j]);
       waddr += keep ? ENTRY_PITCH : 0u;
@@ -254,19 +280,19 @@ __device__ void select_rank(const Sel& s, bool active, int& n, int T, bool drop,
     int nl = work ? n : 0;
     const int n_before = nl;
     const int nw = warp_max(nl);
-    int cnt, above; float blo, bhi;
-    const bool valid = lin_level(s, nl, nw, lo, hi, rank, drop, cnt, above, blo, bhi);
+    BinInfo bi;
+    const bool valid = lin_level(s, nl, nw, lo, hi, rank, drop, bi);
     if (work) {
       if (!valid) { fallback = true; done = true; }
       else {
         n = nl;
-        rank -= above;
-        if (blo == bhi) { s_T = blo; need = rank; exact = true; done = true; }
-        else if (fit_limit >= 0 && n <= fit_limit && n < n_before) { s_T = blo; done = true; }
+        rank -= bi.above;
+        if (fit_limit >= 0 && n <= fit_limit && n < n_before) { s_T = bi.mn1; done = true; }
+        else if (bi.resolve(rank, s_T, need)) { exact = true; done = true; }
         else {
-          // zoom into [blo, bhi]; with drop the entries above stay in the buffer, so the
-          // rank inside the bin is what remains to be resolved
-          lo = blo; hi = bhi;
+          // zoom into the bin; with drop the entries above stay in the buffer, so the rank
+          // inside the bin is what remains to be resolved
+          lo = bi.mn1; hi = bi.mx1;
         }
       }
     }
@@ -313,25 +339,44 @@ struct RowState {
 };
 
 // Re-tightening with a PERSISTENT histogram: the row's score->bin map is fixed at its first
-// re-tightening (NB equal bins over the range seen so far; later, larger scores fall into the
-// top bin), so each call only has to bin the entries appended since the previous call, find
-// the bin b* of rank `keep` from the top, and drop the entries below b* (stable, in place).
-// Bins below b* keep stale counts, which is harmless: the threshold only rises.  If b* is too
-// crowded for the buffer to fit `fit_limit`, score-domain zoom levels finish the job and the
-// histogram is rebuilt at the next call.
-// fit_limit < 0 asks for the exact cut at rank `keep` (n becomes exactly keep).
-__device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_limit, RowState& st) {
-  // (1) map + binning of the new entries
+// re-tightening, so each call only has to bin the entries appended since the previous call,
+// find the bin b* of rank `keep` from the top, and drop the entries below b* (stable, in
+// place).  Bins below b* keep stale counts, which is harmless: the threshold only rises.  If
+// b* is too crowded for the buffer to fit `fit_limit`, the cut is finished inside b* (directly
+// when b* has at most 4 entries, else by score-domain zoom levels) and the histogram is
+// rebuilt at the next call.
+// FINAL: the last call of a row.  The cut is made exact (n becomes `keep`), and the same
+// level also locates rank `kk` (the route / near-miss split): s_k and need_k are returned.
+template <bool FINAL>
+__device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_limit, RowState& st,
+                          int kk, float& s_k, int& need_k) {
+  // (1) map (first call) + binning of the new entries.  With d = mean - min of the buffered
+  // scores the map covers [mean - 0.5 d, mean + 1.3 d]: the cut lies around or above the mean,
+  // and a few far outliers (e.g. a row's own cluster) would otherwise stretch the bins;
+  // whatever falls outside lands in the first / last bin.
   const bool fresh = active && st.binned < 0;
-  if (fresh) {
-    st.map_lo = st.smin;
-    st.map_scale = (float)NB / (st.smax - st.smin);
-    st.binned = 0;
-  }
-  const bool usable = active && st.smax > st.smin && st.map_scale < 1e37f;
   if (__any_sync(FULL, fresh)) {
-    if (fresh) clear_bins(s);
+    const int nf = fresh ? n : 0;
+    const int nwf = warp_max(nf);
+    float sum = 0.f;
+    for (int e0 = 0; e0 < nwf; e0 += BATCH) {
+      float v[BATCH];
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(nf - 1, 0)) * ENTRY_PITCH);
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) sum += e0 + j < nf ? v[j] : 0.f;
+    }
+    if (fresh) {
+      const float mean = sum / (float)max(nf, 1);
+      const float below = 0.5f * (mean - st.smin);
+      const float width = below + fminf(1.3f * (mean - st.smin), st.smax - mean);
+      st.map_lo = mean - below;
+      st.map_scale = (float)NB / width;
+      st.binned = 0;
+      clear_bins(s);
+    }
   }
+  const bool usable = active && st.smax > st.smin && st.map_scale > 0.f && st.map_scale < 1e37f;
   const int from = usable ? st.binned : 0, to = usable ? n : 0;
   const int nw_new = warp_max(to - from);
   const float mlo = st.map_lo, msc = st.map_scale;
@@ -348,13 +393,15 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       aux_st(a, aux_ld(a) + (in ? 1u : 0u));
     }
   }
-  // (2) bin of rank keep, drop what lies below it
-  int bsel, cnt, above;
-  scan_bins(s, keep, bsel, cnt, above);
+  // (2) bin of rank keep (and of rank kk), drop what lies below the former
+  BinInfo bc, bk;
+  int bsel, bsel_k = 0;
+  scan_bins(s, keep, bsel, bc.cnt, bc.above);
+  if (FINAL) scan_bins(s, kk, bsel_k, bk.cnt, bk.above);
+  bc.reset(); bk.reset();
   const int nd = usable ? n : 0;
   const int nw = warp_max(nd);
   uint32_t waddr = s.buf;
-  float blo = __int_as_float(0x7f800000), bhi = __int_as_float(0xff800000);   // bounds of bin b*
   for (int e0 = 0; e0 < nw; e0 += BATCH) {
     float v[BATCH]; uint32_t id[BATCH];
 #pragma unroll
@@ -364,8 +411,9 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     for (int j = 0; j < BATCH; ++j) {
       const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
       const bool live = e0 + j < nd;
-      const bool keep_it = live & (b >= bsel), tgt = live & (b == bsel);
-      blo = fminf(blo, tgt ? v[j] : blo); bhi = fmaxf(bhi, tgt ? v[j] : bhi);
+      const bool keep_it = live & (b >= bsel);
+      bc.track(live & (b == bsel), v[j]);
+      if (FINAL) bk.track(live & (b == bsel_k), v[j]);
       st_entry_if(keep_it, waddr, v[j], id[j]);
       waddr += keep_it ? ENTRY_PITCH : 0u;
     }
@@ -373,26 +421,65 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   if (usable) {
     n = (int)((waddr - s.buf) / ENTRY_PITCH);
     st.binned = n;
-    st.blo = blo; st.tau = blo;       // >= keep seen scores reach blo: a valid threshold
+    st.blo = bc.mn1; st.tau = bc.mn1;  // >= keep seen scores reach mn1: a valid threshold
   }
-  // (3) crowded bin or unusable range: zoom levels / exact cut
+  // (3) crowded bin, unusable range, or the final exact cut: finish inside b*
   const bool more = active && (!usable || n > fit_limit);
-  if (__any_sync(FULL, more)) {
+  float s_T = 0.f; int need = 0;
+  const bool direct = more && usable && bc.resolve(keep - bc.above, s_T, need);
+  const bool zoom = more && !direct;
+#ifdef RR_PHASE_TIMING
+  if (!FINAL) {       // ballots by the whole warp first; only then the lane-0 counters
+    const int nz = __popc(__ballot_sync(FULL, zoom)), nu = __popc(__ballot_sync(FULL, active && !usable));
+    const int ndr = __popc(__ballot_sync(FULL, zoom && bsel == 0));
+    const int ntop = __popc(__ballot_sync(FULL, zoom && bsel == NB - 1));
+    PH_CNT(13, nz); PH_CNT(14, ntop); PH_CNT(15, ndr);
+  }
+#endif
+  if (__any_sync(FULL, zoom)) {
     PH_CNT(9, 1);
-    float s_T; int need; bool exact;
-    // usable: everything left of interest is inside bin b* = [blo, bhi], `above` entries
+    float zs; int zn; bool zexact;
+    // usable: everything left of interest is inside bin b* = [mn1, mx1], `above` entries
     // outrank it; otherwise the whole buffer is searched
-    select_rank(s, more, n, usable ? keep - above : keep, true, fit_limit,
-                usable ? blo : fminf(st.blo, st.smin), usable ? bhi : st.smax, s_T, need, exact);
-    const int w = compact_exact(s, more && exact ? n : 0, s_T, need);
-    if (more) {
-      if (exact) { n = w; st.tau = rr_key_to_float(key_of(s_T) + 1u); }   // later ties lose
-      else st.tau = s_T;
-      st.blo = s_T;
-      // the scratch levels overwrote the bins: rebuild from the buffer at the next call
-      st.binned = usable ? 0 : -1;       // unusable range: choose a new map next time
-      clear_bins(s);
+    select_rank(s, zoom, n, usable ? keep - bc.above : keep, true, fit_limit,
+                usable ? bc.mn1 : fminf(st.blo, st.smin), usable ? bc.mx1 : st.smax, zs, zn, zexact);
+    if (zoom) {
+      if (zexact) { s_T = zs; need = zn; }
+      else { st.tau = zs; st.blo = zs; }        // fits now; zs = smallest surviving score
     }
+    // the scratch levels overwrote the bins of the lanes that zoomed
+    if (zoom) { st.binned = usable ? 0 : -1; clear_bins(s); }
+    const bool cut_exact = direct || (zoom && zexact);
+    const int w = compact_exact(s, cut_exact ? n : 0, s_T, need);
+    if (cut_exact) {
+      n = w;
+      st.tau = rr_key_to_float(key_of(s_T) + 1u);   // later ties have larger ids: they lose
+      st.blo = s_T;
+      if (st.binned > 0) { st.binned = 0; clear_bins(s); }   // counts no longer match
+    }
+  } else if (__any_sync(FULL, direct)) {
+    const int w = compact_exact(s, direct ? n : 0, s_T, need);
+    if (direct) {
+      n = w;
+      st.tau = rr_key_to_float(key_of(s_T) + 1u);
+      st.blo = s_T;
+      if (st.binned > 0) { st.binned = 0; clear_bins(s); }
+    }
+  }
+  // (4) FINAL: the route / near-miss split at rank kk among the `keep` survivors
+  if (FINAL) {
+    const bool split = active && n > kk;
+    float ks = 0.f; int kn = 0;
+    const bool kdirect = split && usable && bk.resolve(kk - bk.above, ks, kn);
+    const bool kzoom = split && !kdirect;
+    if (__any_sync(FULL, kzoom)) {
+      float zs; int zn; bool zexact; int n_ = n;
+      select_rank(s, kzoom, n_, usable ? kk - bk.above : kk, false, -1,
+                  usable ? bk.mn1 : fminf(st.blo, st.smin), usable ? bk.mx1 : st.smax, zs, zn,
+                  zexact);
+      if (kzoom) { ks = zs; kn = zn; }
+    }
+    if (split) { s_k = ks; need_k = kn; }
   }
 }
 
@@ -534,45 +621,50 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       { PH_T0(); ready = mbar_wait(&ctl->acc_full[as], aph, abort_flag); PH_ADD(0); }
       if (!__all_sync(FULL, ready)) { alive = false; break; }
       tc_fence_after();
-#pragma unroll 1
-      for (int c = 0; c < BN / CHUNK; ++c) {
-        const int col0 = t * BN + c * CHUNK;
-        if (col0 >= vmaxw) break;                          // no row of this warp sees these
-        if (__any_sync(FULL, waddr > trigger)) {
-          // re-tighten: raise the threshold until the buffer fits again
+      static_assert(BN == 2 * CHUNK, "a tile is two TMEM loads of 32 columns");
+      if (t * BN < vmaxw) {                                // else: no row of this warp sees it
+        uint32_t acc[2][32];
+        tmem_ld_32x64(tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN, acc[0], acc[1]);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int col0 = t * BN + c * CHUNK;
+          if (col0 >= vmaxw) break;
+          if (__any_sync(FULL, waddr > trigger)) {
+            // re-tighten: raise the threshold until the buffer fits again
+            PH_T0();
+            int n = (int)((waddr - sel.buf) / ENTRY_PITCH);
+            const bool act = n > keep;
+            float dummy_s; int dummy_n;
+            retighten<false>(sel, act, n, keep, (keep + cap - CHUNK) / 2, st, 0, dummy_s, dummy_n);
+            if (act) waddr = sel.buf + (uint32_t)n * ENTRY_PITCH;
+            PH_ADD(1); PH_CNT(8, 1);
+          }
           PH_T0();
-          int n = (int)((waddr - sel.buf) / ENTRY_PITCH);
-          const bool act = n > keep;
-          retighten(sel, act, n, keep, (keep + cap - CHUNK) / 2, st);
-          if (act) waddr = sel.buf + (uint32_t)n * ENTRY_PITCH;
-          PH_ADD(1); PH_CNT(8, 1);
-        }
-        PH_T0();
-        const float tau_f = st.tau;
-        uint32_t acc[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + c * CHUNK, acc);
-        // threshold filter: branch-free appends (predicated stores); waddr is the only chain
-        if (col0 + CHUNK <= vminw) {
+          const float tau_f = st.tau;
+          // threshold filter: branch-free appends (predicated stores); waddr is the only chain
+          if (col0 + CHUNK <= vminw) {
 #pragma unroll
-          for (int q = 0; q < CHUNK; ++q) {
-            const float sc = __uint_as_float(acc[q]) + 0.0f;         // -0.0 -> +0.0
-            const bool pass = sc >= tau_f;
-            st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc);
-            if (pass) st_entry(waddr, sc, (uint32_t)(col0 + q));
-            waddr += pass ? ENTRY_PITCH : 0u;
-          }
-        } else {
+            for (int q = 0; q < CHUNK; ++q) {
+              const float sc = __uint_as_float(acc[c][q]) + 0.0f;         // -0.0 -> +0.0
+              const bool pass = sc >= tau_f;
+              st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc);
+              st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
+              waddr += pass ? ENTRY_PITCH : 0u;
+            }
+          } else {
 #pragma unroll
-          for (int q = 0; q < CHUNK; ++q) {
-            const float sc = __uint_as_float(acc[q]) + 0.0f;
-            const bool valid = col0 + q < v;
-            const bool pass = valid && sc >= tau_f;
-            if (valid) { st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc); }
-            if (pass) st_entry(waddr, sc, (uint32_t)(col0 + q));
-            waddr += pass ? ENTRY_PITCH : 0u;
+            for (int q = 0; q < CHUNK; ++q) {
+              const float sc = __uint_as_float(acc[c][q]) + 0.0f;
+              const bool valid = col0 + q < v;
+              const bool pass = valid && sc >= tau_f;
+              st.smin = fminf(st.smin, valid ? sc : st.smin);
+              st.smax = fmaxf(st.smax, valid ? sc : st.smax);
+              st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
+              waddr += pass ? ENTRY_PITCH : 0u;
+            }
           }
+          PH_ADD(2); PH_CNT(10, 1);
         }
-        PH_ADD(2); PH_CNT(10, 1);
       }
       tc_fence_before();
       mbar_arrive(&ctl->acc_empty[as]);
@@ -583,68 +675,85 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       const int g = have ? (row_list ? row_list[ctl->slot[r]] : ctl->slot[r]) : 0;
       int n = have ? (int)((waddr - sel.buf) / ENTRY_PITCH) : 0;
       PH_CNT(11, 1);
-      // ---- exact cut at rank keep ---------------------------------------------------------------
+      // ---- exact cut at rank keep and split at rank kk (entries <= keep: nothing to cut) ----------
+      float s_k = ninf; int need_k = 0;        // defaults: everything buffered is selected
       {
         PH_T0();
-        const bool cut = n > keep;
-        retighten(sel, cut, n, keep, -1, st);
+        if (__any_sync(FULL, n > kk)) {
+          if (n <= keep) {
+            // rows that see fewer than keep chunks keep everything; only the split remains,
+            // over the whole buffer (no map was ever needed for them)
+          }
+          const bool cut = n > keep;
+          retighten<true>(sel, cut, n, keep, -1, st, kk, s_k, need_k);
+          // rows with kk < n <= keep never enter the cut: split them over the whole buffer
+          const bool small = !cut && n > kk;
+          if (__any_sync(FULL, small)) {
+            float zs; int zn; bool zexact; int n_ = n;
+            select_rank(sel, small, n_, kk, false, -1, st.smin, st.smax, zs, zn, zexact);
+            if (small) { s_k = zs; need_k = zn; }
+          }
+        }
         PH_ADD(3);
-      }
-      // ---- split at rank kk ---------------------------------------------------------------------
-      float s_k = ninf; int need_k = 0;
-      {
-        PH_T0();
-        const bool split = n > kk;
-        int n_ = n; bool exact;
-        select_rank(sel, split, n_, kk, false, -1, fminf(st.blo, st.smin), st.smax, s_k, need_k, exact);
-        if (!split) { s_k = ninf; need_k = 0; }       // everything buffered is selected
-        PH_ADD(4);
       }
       PH_T0();
       for (int w = 0; w < aux_words; ++w) aux_st(sel.aux + w * AUX_PITCH, 0u);   // exclusion bitmap
       int32_t* route = p.routes + (size_t)g * p.k;
       int32_t* sent = p.sentinels + (size_t)g * p.sw;
-      int nr = 0, nn = 0, ties = 0, cur_word = -1;
+      // Pass A (branch-free): classify the survivors.  Route ids are parked in the score word
+      // of slots 0.., near-miss ids in the id word of slots 0.. (a slot is only overwritten
+      // after its entry has been read); the exclusion bitmap is written word by word, which
+      // works because the entries are in ascending chunk id.
+      int nr = 0, nn = 0, ties = 0, cur_word = 0;
       uint32_t cur_bits = 0u;
       float kth = pinf, next = ninf;
       const int nw = warp_max(n);
       for (int e0 = 0; e0 < nw; e0 += BATCH) {
         float sv[BATCH]; uint32_t id[BATCH];
 #pragma unroll
-        for (int j = 0; j < BATCH; ++j) {
-          sv[j] = 0.f; id[j] = 0;
-          if (e0 + j < n) ld_entry(sel.buf + (e0 + j) * ENTRY_PITCH, sv[j], id[j]);
-        }
+        for (int j = 0; j < BATCH; ++j)
+          ld_entry(sel.buf + min(e0 + j, max(n - 1, 0)) * ENTRY_PITCH, sv[j], id[j]);
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
-          if (e0 + j < n) {
-            const bool eq = sv[j] == s_k;
-            const bool in_route = sv[j] > s_k || (eq && ties < need_k);
-            ties += eq;
-            bool excluded = in_route;
-            if (in_route) {
-              route[nr++] = (int)id[j]; kth = fminf(kth, sv[j]);
-            } else {
-              next = fmaxf(next, sv[j]);
-              if (nn < p.m) { sent[nn++] = (int)id[j]; excluded = true; }
-            }
-            // entries are in ascending chunk id: a bitmap word is complete when the id moves
-            // past it, so it is written once, with no read-modify-write
-            const int wi = (int)(id[j] >> 5);
-            if (wi != cur_word) {
-              if (cur_word >= 0) aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
-              cur_word = wi; cur_bits = 0u;
-            }
-            cur_bits |= excluded ? 1u << (id[j] & 31) : 0u;
-          }
+          const bool live = e0 + j < n;
+          const bool eq = live & (sv[j] == s_k);
+          const bool in_route = live & ((sv[j] > s_k) | (eq & (ties < need_k)));
+          const bool in_near = live & !in_route & (nn < p.m);
+          ties += eq;
+          kth = fminf(kth, in_route ? sv[j] : kth);
+          next = fmaxf(next, (live & !in_route) ? sv[j] : next);
+          asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                       ::"r"(sel.buf + nr * ENTRY_PITCH), "r"(id[j]), "r"((uint32_t)in_route) : "memory");
+          asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                       ::"r"(sel.buf + nn * ENTRY_PITCH + 4u), "r"(id[j]), "r"((uint32_t)in_near) : "memory");
+          nr += in_route; nn += in_near;
+          const int wi = live ? (int)(id[j] >> 5) : cur_word;
+          const bool flush = wi != cur_word;
+          asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                       ::"r"(sel.aux + cur_word * AUX_PITCH), "r"(cur_bits), "r"((uint32_t)flush) : "memory");
+          cur_bits = flush ? 0u : cur_bits;
+          cur_word = wi;
+          cur_bits |= (in_route | in_near) ? 1u << (id[j] & 31) : 0u;
         }
       }
-      if (cur_word >= 0) aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
+      aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
       PH_ADD(5);
       if (have) {
         PH_T0();
-        for (int e = nr; e < p.k; ++e) route[e] = -1;
-        for (int e = nn; e < p.m; ++e) sent[e] = -1;
+        // Pass B: copy out, 16 bytes at a time where the row is 16-byte aligned
+        if ((p.k & 3) == 0) {
+          for (int q = 0; q < p.k; q += 4) {
+            int4 o;
+            o.x = q + 0 < nr ? (int)aux_ld(sel.buf + (q + 0) * ENTRY_PITCH) : -1;
+            o.y = q + 1 < nr ? (int)aux_ld(sel.buf + (q + 1) * ENTRY_PITCH) : -1;
+            o.z = q + 2 < nr ? (int)aux_ld(sel.buf + (q + 2) * ENTRY_PITCH) : -1;
+            o.w = q + 3 < nr ? (int)aux_ld(sel.buf + (q + 3) * ENTRY_PITCH) : -1;
+            *reinterpret_cast<int4*>(route + q) = o;
+          }
+        } else {
+          for (int e = 0; e < p.k; ++e) route[e] = e < nr ? (int)aux_ld(sel.buf + e * ENTRY_PITCH) : -1;
+        }
+        for (int e = 0; e < p.m; ++e) sent[e] = e < nn ? (int)aux_ld(sel.buf + e * ENTRY_PITCH + 4u) : -1;
         p.kth[g] = kth;
         p.margin[g] = v > kk ? kth - next : pinf;
 
