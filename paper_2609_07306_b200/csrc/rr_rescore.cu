@@ -54,6 +54,7 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
   const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
   int my_flagged = 0;
   unsigned long long my_cand = 0, my_full = 0;
+  const float err_scale = 4.0f * (float)p.d * 5.9604645e-8f;     // 2 sides x safety 2
 
   const int row_end = min(p.n_q, (tile + 1) * RR_ROW_TILE);
   for (int i = tile * RR_ROW_TILE + warp; i < row_end; i += WARPS) {
@@ -63,7 +64,7 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
     Vec16<T>::load(qc + (size_t)g * p.d + sub * N, q);
     const int32_t* route = p.routes + (size_t)g * p.k;
     const int32_t* sent = p.sentinels + (size_t)g * p.sw;
-    float amin = pinf, bmax = ninf;
+    float amin = pinf, bmax = ninf, nmin = pinf;   // nmin: safe floor of route+near-miss scores
     int n_valid = 0;
     bool bad = false;
     for (int s0 = 0; s0 < p.c; s0 += CPI) {
@@ -72,17 +73,26 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
       if (slot < p.k) idx = route[slot];
       else if (slot < p.c) idx = sent[slot - p.k];
       if (idx >= v) { bad = true; idx = -1; }
-      float acc = 0.f;
+      float acc = 0.f, mag = 0.f;            // mag = sum |q_t k_t|: scale of the rounding error
       if (idx >= 0) {
         float kv[8];
         Vec16<T>::load(kbase + (size_t)idx * p.d + sub * N, kv);
 #pragma unroll
-        for (int e = 0; e < N; ++e) acc = fmaf(q[e], kv[e], acc);
+        for (int e = 0; e < N; ++e) {
+          acc = fmaf(q[e], kv[e], acc);
+          mag = fmaf(fabsf(q[e]), fabsf(kv[e]), mag);
+        }
       }
 #pragma unroll
-      for (int off = LPC / 2; off; off >>= 1) acc += __shfl_xor_sync(FULL, acc, off);
+      for (int off = LPC / 2; off; off >>= 1) {
+        acc += __shfl_xor_sync(FULL, acc, off);
+        mag += __shfl_xor_sync(FULL, mag, off);
+      }
       if (idx >= 0) {
         if (slot < p.k) amin = fminf(amin, acc); else bmax = fmaxf(bmax, acc);
+        // lower bound of this candidate's score under ANY fp32 summation order (the refresh
+        // recomputes it on the tensor cores): |error| <= d * 2^-24 * sum|q_t k_t| per side
+        if (slot < p.k + p.m) nmin = fminf(nmin, acc - err_scale * mag);
         if (sub == 0) ++n_valid;
       }
       if (p.debug && sub == 0 && slot < p.c)
@@ -92,6 +102,7 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
     for (int off = 16; off; off >>= 1) {
       amin = fminf(amin, __shfl_xor_sync(FULL, amin, off));
       bmax = fmaxf(bmax, __shfl_xor_sync(FULL, bmax, off));
+      nmin = fminf(nmin, __shfl_xor_sync(FULL, nmin, off));
       n_valid += __shfl_xor_sync(FULL, n_valid, off);
     }
     if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
@@ -101,6 +112,11 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
       p.flags[g] = flag ? 1 : 0;
       p.alpha[g] = amin;
       p.beta[g] = bmax;
+      // Warm start for the refresh: the route and near-miss candidates are k+m distinct
+      // chunks, so at least k+m scores of this row reach the floor of their current scores
+      // -- a valid (inclusive) lower bound for everything the new route and near-miss set
+      // can contain.
+      p.tau[g] = p.m > 0 ? nmin : ninf;
       my_flagged += flag;
       my_cand += (unsigned long long)n_valid;
       if (flag) my_full += (unsigned long long)v;

@@ -119,9 +119,9 @@ __device__ unsigned long long g_phase[16];
 
 __device__ __forceinline__ int warp_max(int x) { return __reduce_max_sync(FULL, x); }
 
-// order-preserving key of a canonical (no -0.0) score
+// order-preserving key of a score (-0.0 and +0.0 share a key; float compares already agree)
 __device__ __forceinline__ uint32_t key_of(float s) {
-  const uint32_t u = __float_as_uint(s);
+  const uint32_t u = __float_as_uint(s + 0.0f);           // -0.0 -> +0.0
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
@@ -333,7 +333,7 @@ __device__ __forceinline__ int compact_exact(const Sel& s, int n, float s_T, int
 struct RowState {
   float tau;          // pass threshold of the filter (inclusive)
   float blo;          // lower bound of the buffered scores
-  float smin, smax;   // bounds of all valid scores seen
+  float smin, smax;   // smallest buffered score so far / largest valid score seen
   float map_lo, map_scale;   // fixed score -> bin map of the persistent histogram
   int binned;         // buffer entries [0, binned) are counted in the histogram; -1: no map yet
 };
@@ -368,8 +368,12 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     }
     if (fresh) {
       const float mean = sum / (float)max(nf, 1);
-      const float below = 0.5f * (mean - st.smin);
-      const float width = below + fminf(1.3f * (mean - st.smin), st.smax - mean);
+      const float d = mean - st.smin;
+      // full distribution buffered (no threshold yet): skip its lower tail; a buffer that was
+      // filtered from the start (warm threshold) is a truncated upper tail: start at its floor
+      const bool truncated = st.tau > __int_as_float(0xff800000);
+      const float below = truncated ? d : 0.5f * d;
+      const float width = below + fminf((truncated ? 1.5f : 1.3f) * d, st.smax - mean);
       st.map_lo = mean - below;
       st.map_scale = (float)NB / width;
       st.binned = 0;
@@ -402,6 +406,8 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   const int nd = usable ? n : 0;
   const int nw = warp_max(nd);
   uint32_t waddr = s.buf;
+  // bin >= bsel  <=>  (v - lo) * scale >= bsel for bsel >= 1; bin 0 also holds what lies below lo
+  const float tb = bsel == 0 ? __int_as_float(0xff800000) : (float)bsel;
   for (int e0 = 0; e0 < nw; e0 += BATCH) {
     float v[BATCH]; uint32_t id[BATCH];
 #pragma unroll
@@ -409,11 +415,16 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
-      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+      const float t = (v[j] - mlo) * msc;
       const bool live = e0 + j < nd;
-      const bool keep_it = live & (b >= bsel);
-      bc.track(live & (b == bsel), v[j]);
-      if (FINAL) bk.track(live & (b == bsel_k), v[j]);
+      const bool keep_it = live & (t >= tb);
+      if (FINAL) {
+        const int b = max(0, min(NB - 1, __float2int_rz(t)));
+        bc.track(live & (b == bsel), v[j]);
+        bk.track(live & (b == bsel_k), v[j]);
+      } else {
+        bc.mn1 = fminf(bc.mn1, keep_it ? v[j] : bc.mn1);      // smallest survivor
+      }
       st_entry_if(keep_it, waddr, v[j], id[j]);
       waddr += keep_it ? ENTRY_PITCH : 0u;
     }
@@ -426,7 +437,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   // (3) crowded bin, unusable range, or the final exact cut: finish inside b*
   const bool more = active && (!usable || n > fit_limit);
   float s_T = 0.f; int need = 0;
-  const bool direct = more && usable && bc.resolve(keep - bc.above, s_T, need);
+  const bool direct = FINAL && more && usable && bc.resolve(keep - bc.above, s_T, need);
   const bool zoom = more && !direct;
 #ifdef RR_PHASE_TIMING
   if (!FINAL) {       // ballots by the whole warp first; only then the lane-0 counters
@@ -439,10 +450,12 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   if (__any_sync(FULL, zoom)) {
     PH_CNT(9, 1);
     float zs; int zn; bool zexact;
-    // usable: everything left of interest is inside bin b* = [mn1, mx1], `above` entries
-    // outrank it; otherwise the whole buffer is searched
-    select_rank(s, zoom, n, usable ? keep - bc.above : keep, true, fit_limit,
-                usable ? bc.mn1 : fminf(st.blo, st.smin), usable ? bc.mx1 : st.smax, zs, zn, zexact);
+    // FINAL and usable: everything left of interest is inside bin b* = [mn1, mx1] and `above`
+    // entries outrank it; otherwise the whole (already reduced) buffer is searched
+    const bool inbin = FINAL && usable;
+    select_rank(s, zoom, n, inbin ? keep - bc.above : keep, true, fit_limit,
+                inbin ? bc.mn1 : (usable ? bc.mn1 : fminf(st.blo, st.smin)),
+                inbin ? bc.mx1 : st.smax, zs, zn, zexact);
     if (zoom) {
       if (zexact) { s_T = zs; need = zn; }
       else { st.tau = zs; st.blo = zs; }        // fits now; zs = smallest surviving score
@@ -498,8 +511,10 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   uint8_t* s_aux = s_buf + (size_t)cap * ENTRY_PITCH;                 // [aux_words][BM] words
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // Row tiles are handed out heaviest first (under the causal mask the last tile of a problem
+  // walks the most key chunks), so the tail of the grid is made of the short ones.
   const int tiles_m = p.tiles_per_problem;
-  const int prob = blockIdx.x / tiles_m, tm = blockIdx.x % tiles_m;
+  const int prob = blockIdx.x % p.P, tm = tiles_m - 1 - blockIdx.x / p.P;
 
   int seg_lo = 0, seg_hi = p.n_q;
   if (row_list) { seg_lo = p.problem_offsets[prob]; seg_hi = p.problem_offsets[prob + 1]; }
@@ -603,7 +618,9 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     const Sel sel{smem_u32(s_buf) + r * 8u, smem_u32(s_aux) + r * 4u};
     const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
     RowState st;
-    st.tau = row >= 0 ? ninf : pinf;          // padding rows pass nothing
+    // rows of a refresh list start from the threshold the rescoring kernel derived from the
+    // old candidates' current scores (a valid lower bound); anchors start from -inf
+    st.tau = row >= 0 ? (row_list ? p.tau[row_list[ctl->slot[r]]] : ninf) : pinf;   // padding rows pass nothing
     st.blo = pinf; st.smin = pinf; st.smax = ninf;
     st.map_lo = 0.f; st.map_scale = 0.f; st.binned = -1;
     uint32_t waddr = sel.buf;                 // next free entry
@@ -645,19 +662,19 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           if (col0 + CHUNK <= vminw) {
 #pragma unroll
             for (int q = 0; q < CHUNK; ++q) {
-              const float sc = __uint_as_float(acc[c][q]) + 0.0f;         // -0.0 -> +0.0
+              const float sc = __uint_as_float(acc[c][q]);
               const bool pass = sc >= tau_f;
-              st.smin = fminf(st.smin, sc); st.smax = fmaxf(st.smax, sc);
+              st.smin = fminf(st.smin, pass ? sc : st.smin); st.smax = fmaxf(st.smax, sc);
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
               waddr += pass ? ENTRY_PITCH : 0u;
             }
           } else {
 #pragma unroll
             for (int q = 0; q < CHUNK; ++q) {
-              const float sc = __uint_as_float(acc[c][q]) + 0.0f;
+              const float sc = __uint_as_float(acc[c][q]);
               const bool valid = col0 + q < v;
               const bool pass = valid && sc >= tau_f;
-              st.smin = fminf(st.smin, valid ? sc : st.smin);
+              st.smin = fminf(st.smin, pass ? sc : st.smin);
               st.smax = fmaxf(st.smax, valid ? sc : st.smax);
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
               waddr += pass ? ENTRY_PITCH : 0u;
