@@ -163,7 +163,7 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
         alg = cnt["full_pairs"] * 4 + routed * ledger_row
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
                     alg_per_launch=alg / launches)
-    if kind == "rescore":          # unique bytes: inputs + ledger ids + flags/alpha/beta
+    if kind in ("rescore", "rescore_dense"):   # unique bytes: inputs + ledger ids + flags/alpha/beta
         alg = (layer_calls - n_anchor) * (in_bytes + w.rows * (w.c * 4 + 9))
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
                     alg_per_launch=alg / launches)

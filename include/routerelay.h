@@ -77,7 +77,9 @@ typedef struct rr_config {
   int32_t chunk_tokens;    /* >0: also expand routes to token ranges of this chunk size    */
   int32_t debug_outputs;   /* bit 0: relay also stores every candidate score (tests);
                               bit 1: route through the two-pass path (score rows in scratch
-                              + warp-level TopK) even where the fused kernel applies      */
+                              + warp-level TopK) even where the fused kernel applies;
+                              bit 2: rescore candidates with the gathered FP32 kernel even
+                              where the tensor-core strip kernel applies                  */
 } rr_config;
 
 /* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */
@@ -206,6 +208,7 @@ int rr_compact_flags_noalloc(const uint8_t* dev_flags, int32_t n_problems, int32
 #define RR_KIND_EXPAND       6   /* token-range expansion                                    */
 #define RR_KIND_SCORE_TC     7   /* tcgen05 score GEMM                                       */
 #define RR_KIND_ROUTE_FUSED  8   /* tcgen05 score GEMM fused with TopK + sentinels           */
+#define RR_KIND_RESCORE_DENSE 9  /* candidate rescoring from the tensor-core score strip     */
 #define RR_NUM_KINDS        12
 int rr_profile_begin(rr_ledger* L);
 int rr_profile_end(rr_ledger* L, void* stream, float* total_ms, int64_t* launches);

@@ -125,7 +125,8 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   } else {
     if (!L->anchored) return RR_ERR_STATE;
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
-    LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
+    if (L->dense_rescore) LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, st));
+    else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, st));
     if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
@@ -210,6 +211,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
   L->fused = !(cfg->debug_outputs & 2) && rr_route_fused_supported(p);
+  L->dense_rescore = !(cfg->debug_outputs & 4) && rr_rescore_dense_supported(p);
   *out = L;
   return RR_OK;
 }
@@ -349,6 +351,7 @@ const char* rr_kind_name(int kind) {
     case RR_KIND_EXPAND: return "expand";
     case RR_KIND_SCORE_TC: return "score_tc";
     case RR_KIND_ROUTE_FUSED: return "route_fused";
+    case RR_KIND_RESCORE_DENSE: return "rescore_dense";
     default: return "";
   }
 }

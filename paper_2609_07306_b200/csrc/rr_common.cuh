@@ -36,6 +36,7 @@ struct rr_ledger {
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
   bool fused;                              // full routing runs in the fused tensor-core kernel
+  bool dense_rescore;                      // relay rescoring reads the tensor-core score strip
   unsigned long long dense_pairs_per_layer;
   // benchmark-only per-kernel timing
   bool profiling = false;
@@ -90,6 +91,9 @@ cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int 
                                 cudaStream_t st);
 cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
                               cudaStream_t st);
+bool rr_rescore_dense_supported(const RRParams& p);
+cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
+                                    cudaStream_t st);
 cudaError_t rr_launch_compact(const RRParams& p, cudaStream_t st);
 cudaError_t rr_launch_anchor_fill(const RRParams& p, cudaStream_t st);
 cudaError_t rr_launch_update(const RRParams& p, int is_anchor, unsigned long long dense_pairs,

@@ -25,18 +25,20 @@ def test_tiny_fp32_all_layers():
     parity.assert_clean(rep)
 
 
-@pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
-def test_moderate_bf16_causal_all_layers(two_pass):
-    rep = parity.run_teacher_forced(W.moderate(), two_pass=two_pass)
+@pytest.mark.parametrize("two_pass,gathered", [(False, False), (False, True), (True, True)],
+                         ids=["fused+strip", "fused+gathered", "two_pass+gathered"])
+def test_moderate_bf16_causal_all_layers(two_pass, gathered):
+    rep = parity.run_teacher_forced(W.moderate(), two_pass=two_pass, gathered=gathered)
     _report(rep)
     parity.assert_clean(rep)
 
 
-@pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
+@pytest.mark.parametrize("two_pass,gathered", [(False, False), (False, True), (True, True)],
+                         ids=["fused+strip", "fused+gathered", "two_pass+gathered"])
 @pytest.mark.parametrize("n", [128, 512])
-def test_sweep_shapes(n, two_pass):
+def test_sweep_shapes(n, two_pass, gathered):
     w = W.sweep(n, 0.15).replace(heads=4, layers=4, anchor_every=3)
-    rep = parity.run_teacher_forced(w, two_pass=two_pass)
+    rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
     _report(rep)
     parity.assert_clean(rep)
 
@@ -45,8 +47,8 @@ def test_ragged_shapes_and_wide_ledger():
     # n_q not a multiple of any tile, n_q != n_k, non-causal, d=64 bf16, wide candidate set
     w = W.RouteWorkload("ragged", 1, 3, 200, 333, 64, 12, 24, 12, layers=3, anchor_every=3,
                         dtype=W.DTYPE_BF16, centroids=16, rho=0.05, causal=False, seed=3)
-    for two_pass in (False, True):
-        rep = parity.run_teacher_forced(w, two_pass=two_pass)
+    for two_pass, gathered in ((False, False), (False, True), (True, True)):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
         _report(rep)
         parity.assert_clean(rep)
     w = W.RouteWorkload("ragged32", 2, 1, 130, 130, 128, 5, 0, 7, layers=3, anchor_every=2,
