@@ -58,23 +58,45 @@ struct Ctl {
 constexpr uint32_t ENTRY_PITCH = BM * 8, AUX_PITCH = BM * 4;
 struct Sel { uint32_t buf, aux; };
 
+// Optional self-check (compile with -DRR_BOUNDS_CHECK): a shared-window address beyond the
+// CTA's allocation is recorded (first offender wins) and the access is skipped.
+#ifdef RR_BOUNDS_CHECK
+__device__ unsigned int g_oob[4];
+__device__ __forceinline__ bool oob(uint32_t addr, unsigned code) {
+  if (addr < 233472u) return false;
+  if (atomicCAS(&g_oob[0], 0u, code) == 0u) { g_oob[1] = addr; g_oob[2] = blockIdx.x; g_oob[3] = threadIdx.x; }
+  return true;
+}
+#define RR_OOB(addr, code) if (oob(addr, code)) return
+#define RR_OOB_V(addr, code, val) if (oob(addr, code)) return val
+#else
+#define RR_OOB(addr, code) do {} while (0)
+#define RR_OOB_V(addr, code, val) do {} while (0)
+#endif
+
 __device__ __forceinline__ void st_entry(uint32_t addr, float s, uint32_t id) {
+  RR_OOB(addr, 1);
   asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "f"(s), "r"(id) : "memory");
 }
 __device__ __forceinline__ void ld_entry(uint32_t addr, float& s, uint32_t& id) {
+  s = 0.f; id = 0;
+  RR_OOB(addr, 2);
   asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=f"(s), "=r"(id) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ float ld_score(uint32_t addr) {
+  RR_OOB_V(addr, 3, 0.f);
   float s;
   asm volatile("ld.shared.b32 %0, [%1];" : "=f"(s) : "r"(addr) : "memory");
   return s;
 }
 __device__ __forceinline__ uint32_t aux_ld(uint32_t addr) {
+  RR_OOB_V(addr, 4, 0u);
   uint32_t v;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
   return v;
 }
 __device__ __forceinline__ void aux_st(uint32_t addr, uint32_t v) {
+  RR_OOB(addr, 5);
   asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void aux_inc(uint32_t addr) {
@@ -82,6 +104,7 @@ __device__ __forceinline__ void aux_inc(uint32_t addr) {
 }
 // predicated forms: no branch is emitted, the access is simply masked off
 __device__ __forceinline__ void st_entry_if(bool pred, uint32_t addr, float s, uint32_t id) {
+  if (pred) { RR_OOB(addr, 6); }
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.shared.v2.b32 [%0], {%1, %2};\n\t}"
                ::"r"(addr), "f"(s), "r"(id), "r"((uint32_t)pred) : "memory");
 }
@@ -508,7 +531,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   uint8_t* sB = smem + C::A_BYTES;
   Ctl* ctl = (Ctl*)(smem + C::A_BYTES + B_STAGES * C::B_BYTES);
   uint8_t* s_buf = (uint8_t*)ctl + C::CTL_BYTES;                      // [cap][BM] 8-byte entries
-  uint8_t* s_aux = s_buf + (size_t)cap * ENTRY_PITCH;                 // [aux_words][BM] words
+  uint8_t* s_aux = s_buf + (size_t)cap * ENTRY_PITCH;                 // [NB][BM] histogram words
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // Row tiles are handed out heaviest first (under the causal mask the last tile of a problem
@@ -714,7 +737,17 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         PH_ADD(3);
       }
       PH_T0();
-      for (int w = 0; w < aux_words; ++w) aux_st(sel.aux + w * AUX_PITCH, 0u);   // exclusion bitmap
+      // exclusion bitmap: in the thread's histogram words when they suffice, else in the tail of
+      // the thread's OWN buffer column (entries beyond keep are dead after the final cut; two
+      // words per entry slot).  Other warps may still be filtering, so nothing outside this
+      // thread's column may be touched.
+      const bool tail = aux_words > NB;
+      const uint32_t bm_base = tail ? sel.buf + (uint32_t)keep_cfg * ENTRY_PITCH : sel.aux;
+      auto bm = [&](int w) -> uint32_t {
+        return tail ? bm_base + (uint32_t)(w >> 1) * ENTRY_PITCH + (uint32_t)(w & 1) * 4u
+                    : bm_base + (uint32_t)w * AUX_PITCH;
+      };
+      for (int w = 0; w < aux_words; ++w) aux_st(bm(w), 0u);
       int32_t* route = p.routes + (size_t)g * p.k;
       int32_t* sent = p.sentinels + (size_t)g * p.sw;
       // Pass A (branch-free): classify the survivors.  Route ids are parked in the score word
@@ -747,13 +780,13 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           const int wi = live ? (int)(id[j] >> 5) : cur_word;
           const bool flush = wi != cur_word;
           asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
-                       ::"r"(sel.aux + cur_word * AUX_PITCH), "r"(cur_bits), "r"((uint32_t)flush) : "memory");
+                       ::"r"(bm(cur_word)), "r"(cur_bits), "r"((uint32_t)flush) : "memory");
           cur_bits = flush ? 0u : cur_bits;
           cur_word = wi;
           cur_bits |= (in_route | in_near) ? 1u << (id[j] & 31) : 0u;
         }
       }
-      aux_st(sel.aux + cur_word * AUX_PITCH, cur_bits);
+      aux_st(bm(cur_word), cur_bits);
       PH_ADD(5);
       if (have) {
         PH_T0();
@@ -784,13 +817,13 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
             const int limit = 64 * p.r;
             for (int t = 0; t < limit && taken < p.r; ++t) {
               const int j = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)t), (uint32_t)v);
-              const uint32_t wa = sel.aux + (j >> 5) * AUX_PITCH;
+              const uint32_t wa = bm(j >> 5);
               const uint32_t w = aux_ld(wa), bit = 1u << (j & 31);
               if (!(w & bit)) { aux_st(wa, w | bit); rnd[taken++] = j; }
             }
           }
           for (int j = 0; j < v && taken < p.r; ++j)
-            if (!((aux_ld(sel.aux + (j >> 5) * AUX_PITCH) >> (j & 31)) & 1u)) rnd[taken++] = j;
+            if (!((aux_ld(bm(j >> 5)) >> (j & 31)) & 1u)) rnd[taken++] = j;
         }
         for (int e = taken; e < p.r; ++e) rnd[e] = -1;
         PH_ADD(6);
@@ -811,22 +844,29 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 bool plan(const RRParams& p, int& cap, int& aux_words, size_t& smem_bytes) {
   const int keep = p.k + (p.m > 0 ? p.m : 1);
   const size_t fixed = p.d == 128 ? Cfg<128>::FIXED_BYTES : Cfg<64>::FIXED_BYTES;
-  aux_words = (p.n_k + 31) / 32;
-  if (aux_words < NB) aux_words = NB;
+  aux_words = (p.n_k + 31) / 32;                 // words of the exclusion bitmap
   const size_t max_smem = 227 * 1024;
-  const size_t aux = (size_t)aux_words * BM * 4;
-  if (fixed + aux >= max_smem) return false;
-  const size_t per_entry = ENTRY_PITCH;
-  int fit = (int)((max_smem - fixed - aux) / per_entry);
+  const size_t hist = (size_t)NB * AUX_PITCH;
+  if (fixed + hist >= max_smem) return false;
+  const int fit = (int)((max_smem - fixed - hist) / ENTRY_PITCH);
   cap = keep + 96;
   if (cap > fit) cap = fit;
   if (cap < keep + CHUNK) return false;
+  // a bitmap wider than the histogram lives in the buffer entries beyond `keep`
+  if (aux_words > NB && (aux_words + 1) / 2 > cap - keep) return false;
   if (p.n_k > 65535) return false;
-  smem_bytes = fixed + aux + (size_t)cap * per_entry;
+  smem_bytes = fixed + hist + (size_t)cap * ENTRY_PITCH;
   return true;
 }
 
 }  // namespace
+
+#ifdef RR_BOUNDS_CHECK
+extern "C" int rr_debug_oob(unsigned int* out4) {
+  cudaDeviceSynchronize();
+  return cudaMemcpyFromSymbol(out4, g_oob, 16) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 #ifdef RR_PHASE_TIMING
 extern "C" int rr_debug_phase_counters(unsigned long long* out16, int reset) {

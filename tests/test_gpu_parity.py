@@ -58,6 +58,35 @@ def test_ragged_shapes_and_wide_ledger():
     parity.assert_clean(rep)
 
 
+def test_long_context_shape_small():
+    # n_k = 2048, k = 64, 32 + 32 sentinels (c = 128), token ranges; 2 heads, 3 layers
+    w = W.long_ctx().replace(batch=1, heads=2, layers=3, anchor_every=2)
+    for two_pass, gathered in ((False, False), (True, True)):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
+        _report(rep)
+        parity.assert_clean(rep)
+
+
+def test_high_drift_full_size_sampled_problems():
+    """BASELINE configuration 4 at full size (256 problems x 1024 rows, the launch the
+    benchmark times), first 5 layers (anchor, 3 relays, relay after a centroid re-draw);
+    three problems are checked row by row against the oracle, the integer work (compaction,
+    ages, stable rows) on all 262144 rows."""
+    w = W.high_drift()
+    rep = parity.run_teacher_forced(w, check_problems=[0, 101, 255], layers=5, gen_threads=16)
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_long_context_full_size_sampled_problems():
+    """BASELINE configuration 5 at full size (64 problems x 2048 rows), 3 layers, two
+    problems checked against the oracle."""
+    w = W.long_ctx()
+    rep = parity.run_teacher_forced(w, check_problems=[3, 60], layers=3, gen_threads=16)
+    _report(rep)
+    parity.assert_clean(rep)
+
+
 def test_degenerate_all_equal_scores():
     """All-zero inputs: every score ties; TopK must take the smallest ids, margin 0, and the
     challenge test (tie => flagged) must flag every row that has a sentinel."""
