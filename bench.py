@@ -220,6 +220,8 @@ def run_ours(args) -> None:
         return float(t.item())
 
     w = _workload(args.workload).replace(seed=rank)      # weak scaling: own problems per rank
+    if args.layers:
+        w = w.replace(layers=min(args.layers, w.layers))
     L = w.layers
     peaks = _peaks()
     esz = 2 if w.dtype == W.DTYPE_BF16 else 4
@@ -237,7 +239,8 @@ def run_ours(args) -> None:
     if w.dtype == W.DTYPE_BF16:
         dq, dk = dq.view(torch.bfloat16), dk.view(torch.bfloat16)
 
-    led = RouteLedger(config_from_workload(w), device=str(dev))
+    cfg = config_from_workload(w, two_pass=args.two_pass, gathered=args.gathered)
+    led = RouteLedger(cfg, device=str(dev))
     stream = torch.cuda.current_stream(dev)
 
     def step():
@@ -264,6 +267,17 @@ def run_ours(args) -> None:
     clock_info = clocks.stop()
     ms_per_step = ms_total / args.steps
     value = w.rows * L * world / (ms_per_step * 1e-3)
+    if args.profile_only:            # short run for profiler captures: no extra passes
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup,
+                              "ms_per_step": ms_per_step, "gpu_launches": int(launches),
+                              "config": {"workload": w.name, "layers": L},
+                              "note": "profile-only run"}))
+        led.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- per-kernel device times (same steps, events around every launch) ---------------
     led.reset()
@@ -304,7 +318,7 @@ def run_ours(args) -> None:
     layer_ms = [statistics.median(r[l] for r in reps) for l in range(L)]
     anchor_ms = statistics.median(layer_ms[l] for l in range(L) if w.is_anchor(l))
     relay_ms = statistics.median(layer_ms[l] for l in range(L) if not w.is_anchor(l))
-    full_led = RouteLedger(config_from_workload(w), device=str(dev))
+    full_led = RouteLedger(cfg, device=str(dev))
     freps = [per_layer_ms(lambda l: full_led.route_anchor(dq[l], dk[l], l)) for _ in range(3)]
     full_ms = statistics.median(statistics.median(r[l] for r in freps) for l in range(L))
 
@@ -350,7 +364,7 @@ def run_ours(args) -> None:
     # ---- CPU oracle beside it (rank 0, N = 1 only) -----------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, dt, summ, sample = _oracle_sample(w, 4, 9)
+        v, dt, summ, sample = _oracle_sample(w, 12, 9)
         cpu = {"value": v, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
                "sample": sample, "oracle_recall": summ.recall_all,
                "oracle_flagged_fraction": summ.flagged_relay_fraction}
@@ -394,6 +408,13 @@ def main():
     ap.add_argument("--workload", default="high_drift",
                     choices=sorted(W.PRESETS) + ["sweep1024"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="truncate the layer schedule")
+    ap.add_argument("--profile-only", action="store_true",
+                    help="warm-up + timed steps only (for profiler captures)")
+    ap.add_argument("--two-pass", action="store_true",
+                    help="route through score rows in scratch + warp-level TopK")
+    ap.add_argument("--gathered", action="store_true",
+                    help="rescore candidates with the gathered FP32 kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -54,6 +54,24 @@ int validate(const rr_config* c) {
   return RR_OK;
 }
 
+// RRParams fields that decide which kernels apply (host-only; no pointers).
+RRParams shape_params(const rr_config* cfg) {
+  RRParams p{};
+  p.P = cfg->batch * cfg->heads; p.n_q = cfg->n_q; p.n_k = cfg->n_k; p.d = cfg->d;
+  p.k = cfg->k; p.m = cfg->m; p.r = cfg->r; p.sw = cfg->m + cfg->r; p.c = cfg->k + p.sw;
+  p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
+  p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs & 1;
+  p.rows = p.P * p.n_q;
+  p.tiles_per_problem = (p.n_q + RR_ROW_TILE - 1) / RR_ROW_TILE;
+  p.n_tiles = p.P * p.tiles_per_problem;
+  p.gamma = cfg->gamma; p.seed = cfg->seed;
+  return p;
+}
+
+bool uses_fused(const rr_config* cfg) {
+  return !(cfg->debug_outputs & 2) && rr_route_fused_supported(shape_params(cfg));
+}
+
 Layout make_layout(const rr_config* c) {
   Layout L{};
   const size_t P = (size_t)c->batch * c->heads, rows = P * c->n_q;
@@ -80,7 +98,8 @@ Layout make_layout(const rr_config* c) {
   L.status = o;          o = align_up(o + 4);
   L.token_ranges = o;    o = align_up(o + (c->chunk_tokens > 0 ? rows * c->k * 8 : 0));
   L.cand_scores = o;     o = align_up(o + ((c->debug_outputs & 1) ? rows * cw * 4 : 0));
-  L.S = o;               o = align_up(o + rows * (size_t)c->n_k * 4);
+  // score rows are only materialised by the two-pass path
+  L.S = o;               o = align_up(o + (uses_fused(c) ? 0 : rows * (size_t)c->n_k * 4));
   L.scratch_total = o;
   return L;
 }
@@ -187,14 +206,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   cudaGetLastError();
   L->dense_pairs_per_layer = dense_pairs(cfg);
   RRParams& p = L->p;
-  p.P = cfg->batch * cfg->heads; p.n_q = cfg->n_q; p.n_k = cfg->n_k; p.d = cfg->d;
-  p.k = cfg->k; p.m = cfg->m; p.r = cfg->r; p.sw = cfg->m + cfg->r; p.c = cfg->k + p.sw;
-  p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
-  p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs & 1;
-  p.rows = p.P * p.n_q;
-  p.tiles_per_problem = (p.n_q + RR_ROW_TILE - 1) / RR_ROW_TILE;
-  p.n_tiles = p.P * p.tiles_per_problem;
-  p.gamma = cfg->gamma; p.seed = cfg->seed;
+  p = shape_params(cfg);
   char* lb = (char*)dev_ledger; char* sb = (char*)dev_scratch;
   p.routes = (int32_t*)(lb + lay.routes); p.sentinels = (int32_t*)(lb + lay.sentinels);
   p.ages = (int32_t*)(lb + lay.ages); p.kth = (float*)(lb + lay.kth);
@@ -210,7 +222,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.token_ranges = cfg->chunk_tokens > 0 ? (int32_t*)(sb + lay.token_ranges) : nullptr;
   p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
-  L->fused = !(cfg->debug_outputs & 2) && rr_route_fused_supported(p);
+  L->fused = uses_fused(cfg);
   L->dense_rescore = !(cfg->debug_outputs & 4) && rr_rescore_dense_supported(p);
   *out = L;
   return RR_OK;

@@ -54,7 +54,9 @@ def test_workspace_sizes():
     lb, sb = B.rr_workspace_bytes(cfg)
     rows = 2 * 256
     assert lb >= rows * (16 + 16 + 3) * 4
-    assert sb >= rows * 256 * 4                      # two-pass score rows
+    assert sb < rows * 256 * 4                       # fused path: no score rows in scratch
+    _, sb2 = B.rr_workspace_bytes(_cfg(debug_outputs=2))
+    assert sb2 >= rows * 256 * 4                     # two-pass path: score rows
     assert B.rr_export_bytes(cfg) == rows * (16 + 16 + 3) * 4
     # paper, Section 4.4: int32 index ledger, n_q = 1024, c = 64 -> 256 KB
     cfg = _cfg(heads=1, n_q=1024, n_k=1024, k=32, m=16, r=16)
