@@ -114,7 +114,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-i", str(gpu_index)],
+                 "-lms", "50", "-i", str(gpu_index)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -146,6 +146,13 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels that
+# dominate a high_drift step, from the ncu captures summarised in profiles/
+# (route_fused_high_drift.md: 199.2 MB anchor / 204.3 MB refresh; rescore_dense_high_drift.md).
+NCU_TRAFFIC_BYTES = {"high_drift": {"route_fused": (4 * 199.2e6 + 28 * 204.3e6) / 32,
+                                    "rescore_dense": 243.9e6}}
+
+
 # ----------------------------------------------------------------------------- roofline
 def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
     """Algorithmic work of one kernel kind over one step, its bound and measured peak.
@@ -175,9 +182,15 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
                     alg_per_launch=alg / launches)
     if kind in ("score_tc", "route_fused"):
         alg = 2.0 * w.d * cnt["full_pairs"]
-        return dict(bound="tensor", achieved=alg / sec / 1e12,
-                    peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
-                    alg_per_launch=alg / launches)
+        out = dict(bound="tensor", achieved=alg / sec / 1e12,
+                   peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                   alg_per_launch=alg / launches)
+        if kind == "route_fused":   # also against HBM: inputs of every routed tile + ledger rows
+            calls = layer_calls
+            alg_b = calls * in_bytes * (routed / (calls * w.rows)) + routed * ledger_row
+            out["hbm_achieved_gbs"] = alg_b / sec / 1e9
+            out["hbm_frac"] = out["hbm_achieved_gbs"] / peaks["hbm_gbs"]
+        return out
     if kind == "compact":
         alg = (layer_calls - n_anchor) * w.rows + cnt["flagged_rows"] * 4
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
@@ -294,12 +307,20 @@ def run_ours(args) -> None:
         kernels[kind] = {"launches_per_step": n // args.steps, "avg_us": 1e3 * ms / n,
                          "share": ms / tot_ms, "bound": r["bound"], "achieved": r["achieved"],
                          "peak": r["peak"], "unit": r["unit"], "frac": r["achieved"] / r["peak"]}
+        if "hbm_frac" in r:
+            kernels[kind]["hbm_achieved_gbs"] = r["hbm_achieved_gbs"]
+            kernels[kind]["hbm_frac"] = r["hbm_frac"]
     top = next(iter(kernels))
     tk = kernels[top]
     roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
                 "peak": tk["peak"], "unit": tk["unit"], "frac": tk["frac"],
-                "peak_source": peaks["source"] if tk["bound"] != "alu" else
-                "148 SMs x 128 FMA/clk x 2 x sampled SM clock", "traffic": None}
+                "peak_source": (peaks["source"] + " (sustained bf16)" if tk["bound"] == "tensor"
+                                else peaks["source"]) if tk["bound"] != "alu" else
+                "148 SMs x 128 FMA/clk x 2 x sampled SM clock",
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(top) if not args.layers else None}
+    if "hbm_frac" in tk:
+        roofline["hbm_achieved_gbs"] = tk["hbm_achieved_gbs"]
+        roofline["hbm_frac"] = tk["hbm_frac"]
 
     # ---- per-layer times: anchor layers, relay layers, and full routing on every layer ---
     def per_layer_ms(fn_of_layer):
@@ -402,7 +423,7 @@ def run_ours(args) -> None:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="high_drift",
