@@ -200,6 +200,31 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
                 alg_per_launch=alg / launches)
 
 
+# ----------------------------------------------------------------------------- multi-GPU plumbing
+def shard_workload(w: W.RouteWorkload, rank: int) -> W.RouteWorkload:
+    """Routing problems are independent (the ledger, the scores and the refresh decisions of a
+    row never cross its batch x head pair), so N GPUs need no exchange on the data path: every
+    rank routes its own batch of problems (weak scaling).  Rank r's batch is the workload with
+    seed r, i.e. different problems on every rank."""
+    return w.replace(seed=int(w.seed) + int(rank))
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """Step time of the job = the slowest rank's device time."""
+    if world == 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_rows_per_s(rows_per_rank: int, layers: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: all ranks' rows x layers over the slowest rank's step time."""
+    return rows_per_rank * layers * world / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args) -> None:
     import torch
@@ -225,14 +250,7 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
-    w = _workload(args.workload).replace(seed=rank)      # weak scaling: own problems per rank
+    w = shard_workload(_workload(args.workload), rank)   # weak scaling: own problems per rank
     if args.layers:
         w = w.replace(layers=min(args.layers, w.layers))
     L = w.layers
@@ -275,11 +293,11 @@ def run_ours(args) -> None:
         step()
     e1.record(stream)
     barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     launches = B.rr_kernel_launch_count() - launches0
     clock_info = clocks.stop()
     ms_per_step = ms_total / args.steps
-    value = w.rows * L * world / (ms_per_step * 1e-3)
+    value = aggregate_rows_per_s(w.rows, L, world, ms_per_step)
     if args.profile_only:            # short run for profiler captures: no extra passes
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
@@ -361,26 +379,37 @@ def run_ours(args) -> None:
     pairs = (c1["cand_pairs"] + c1["full_pairs"]) / c1["dense_pairs"]
     status = led.status()
 
-    # ---- end to end: host buffers through rr_route_layer_host --------------------------------
-    sq = torch.empty_like(dq[0]); sk = torch.empty_like(dk[0])
-    host_routes = torch.empty((w.rows, w.k), dtype=torch.int32).pin_memory()
+    # ---- end to end: host buffers through rr_route_layers_host ------------------------------
+    # (pinned host inputs copied in, every layer's routes copied back, copies overlapped with
+    # the routing on a second stream -- all inside the library call)
+    sq = [torch.empty_like(dq[0]) for _ in range(2)]
+    sk = [torch.empty_like(dk[0]) for _ in range(2)]
+    sr = [torch.empty((w.rows, w.k), dtype=torch.int32, device=dev) for _ in range(2)]
+    host_routes = [torch.empty((w.rows, w.k), dtype=torch.int32).pin_memory() for _ in range(2)]
+    copy_stream = torch.cuda.Stream(dev)
+    d2h_stream = torch.cuda.Stream(dev)
+    anchors = [w.is_anchor(l) for l in range(L)]
 
     def step_e2e():
-        for l in range(L):
-            led.route_layer_host(hq[l], hk[l], sq, sk, l, w.is_anchor(l), host_routes)
+        led.route_layers_host([hq[l] for l in range(L)], [hk[l] for l in range(L)], anchors, 0,
+                              sq, sk, sr, [host_routes[l & 1] for l in range(L)], copy_stream,
+                              d2h_stream)
 
     step_e2e()
     barrier()
     e0.record(stream)
     for _ in range(args.steps):
         step_e2e()
+        stream.wait_stream(copy_stream)        # the step ends when its last routes are on the host
+        stream.wait_stream(d2h_stream)
     e1.record(stream)
     barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     h2d = L * w.problems * (w.n_q + w.n_k) * w.d * esz
     d2h = L * w.rows * w.k * 4
-    e2e = {"value": w.rows * L * world / (ms_e2e * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
+    e2e = {"value": aggregate_rows_per_s(w.rows, L, world, ms_e2e), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
+           "api": "rr_route_layers_host (copies overlapped on a second stream)"}
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) -----------------------------------------
     cpu = None

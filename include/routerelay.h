@@ -144,6 +144,26 @@ int rr_route_layer_host(rr_ledger* L, const void* host_qc, const void* host_kc,
                         void* dev_qc_staging, void* dev_kc_staging, int32_t layer,
                         int32_t is_anchor, int32_t* host_routes, void* stream);
 
+/* A run of consecutive layers driven from HOST buffers, with the copies overlapped with the
+ * routing: layer l's inputs are copied on `copy_stream` into staging set l%2 while layer l-1
+ * runs on `stream`; after each layer its routes are snapshotted device-to-device and copied
+ * to the host on `copy_stream`.
+ *   host_qc / host_kc   [n_layers] host pointers (pinned memory for real overlap), layout as above
+ *   is_anchor           [n_layers] non-zero = anchor layer
+ *   dev_qc_staging / dev_kc_staging   [2] device buffers of one layer's Qc / Kc each
+ *   dev_routes_staging  [2] device buffers of rows*k int32 each (may be NULL if host_routes is)
+ *   host_routes         [n_layers] host pointers (rows*k int32 each) or NULL entries / NULL
+ *   d2h_stream          stream of the route downloads (NULL = copy_stream); a separate one lets
+ *                       uploads and downloads use both directions of the link at once
+ * Enqueue-only: the caller synchronises ALL streams before reading host_routes or reusing
+ * any buffer.  The library creates a few CUDA events on first use (no device memory). */
+int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host_qc,
+                         const void* const* host_kc, const int32_t* is_anchor,
+                         int32_t first_layer, void* const* dev_qc_staging,
+                         void* const* dev_kc_staging, void* const* dev_routes_staging,
+                         int32_t* const* host_routes, void* stream, void* copy_stream,
+                         void* d2h_stream);
+
 /* Device pointers to state and per-layer outputs. */
 int rr_ledger_views(rr_ledger* L, rr_views* out);
 

@@ -78,6 +78,9 @@ def lib() -> C.CDLL:
         L.rr_route_anchor.argtypes = [vp, vp, vp, i32, vp]
         L.rr_route_relay.argtypes = [vp, vp, vp, i32, vp]
         L.rr_route_layer_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.rr_route_layers_host.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), i32,
+                                           C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                           C.POINTER(vp), vp, vp, vp]
         L.rr_ledger_views.argtypes = [vp, C.POINTER(rr_views)]
         L.rr_ledger_export.argtypes = [vp, vp, sz, vp]
         L.rr_ledger_import.argtypes = [vp, vp, sz, vp]
@@ -100,7 +103,7 @@ def lib() -> C.CDLL:
         L.rr_last_cuda_error.restype = C.c_char_p
         for name in ("rr_workspace_bytes", "rr_export_bytes", "rr_ledger_init", "rr_ledger_reset",
                      "rr_ledger_destroy", "rr_route_anchor", "rr_route_relay",
-                     "rr_route_layer_host", "rr_ledger_views", "rr_ledger_export",
+                     "rr_route_layer_host", "rr_route_layers_host", "rr_ledger_views", "rr_ledger_export",
                      "rr_ledger_import", "rr_ledger_status"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -161,6 +164,20 @@ def rr_route_layer_host(h: int, host_qc: int, host_kc: int, dev_qc: int, dev_kc:
     _check(lib().rr_route_layer_host(h, host_qc, host_kc, dev_qc, dev_kc, layer,
                                      1 if is_anchor else 0, host_routes, stream),
            "rr_route_layer_host")
+
+
+def rr_route_layers_host(h: int, host_qc, host_kc, is_anchor, first_layer: int, dev_qc, dev_kc,
+                         dev_routes, host_routes, stream: int, copy_stream: int,
+                         d2h_stream: int = 0) -> None:
+    """host_qc/host_kc/host_routes: sequences of host addresses (one per layer; host_routes may be
+    None); dev_qc/dev_kc/dev_routes: two device addresses each (dev_routes may be None)."""
+    n = len(host_qc)
+    arr = lambda xs: (C.c_void_p * len(xs))(*xs)
+    _check(lib().rr_route_layers_host(
+        h, n, arr(host_qc), arr(host_kc), (C.c_int32 * n)(*[1 if a else 0 for a in is_anchor]),
+        first_layer, arr(dev_qc), arr(dev_kc), arr(dev_routes) if dev_routes else None,
+        arr(host_routes) if host_routes else None, stream, copy_stream, d2h_stream or None),
+           "rr_route_layers_host")
 
 
 def rr_ledger_views(h: int) -> rr_views:

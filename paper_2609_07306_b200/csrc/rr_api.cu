@@ -237,6 +237,9 @@ int rr_ledger_reset(rr_ledger* L, void* stream) {
 
 int rr_ledger_destroy(rr_ledger* L) {
   if (!L) return RR_ERR_INVALID_ARG;
+  for (int b = 0; b < 2; ++b)
+    for (cudaEvent_t e : {L->ev_copied[b], L->ev_consumed[b], L->ev_snap[b], L->ev_d2h[b]})
+      if (e) cudaEventDestroy(e);
   delete L;
   return RR_OK;
 }
@@ -265,6 +268,64 @@ int rr_route_layer_host(rr_ledger* L, const void* host_qc, const void* host_kc,
   if (host_routes)
     RR_CUDA(cudaMemcpyAsync(host_routes, p.routes, (size_t)p.rows * p.k * 4,
                             cudaMemcpyDeviceToHost, st));
+  return RR_OK;
+}
+
+int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host_qc,
+                         const void* const* host_kc, const int32_t* is_anchor,
+                         int32_t first_layer, void* const* dev_qc_staging,
+                         void* const* dev_kc_staging, void* const* dev_routes_staging,
+                         int32_t* const* host_routes, void* stream, void* copy_stream,
+                         void* d2h_stream) {
+  if (!L || n_layers < 0 || !host_qc || !host_kc || !is_anchor || !dev_qc_staging ||
+      !dev_kc_staging || first_layer < 0)
+    return RR_ERR_INVALID_ARG;
+  if (host_routes && !dev_routes_staging) return RR_ERR_INVALID_ARG;
+  for (int b = 0; b < 2; ++b)
+    if (!dev_qc_staging[b] || !dev_kc_staging[b] || (host_routes && !dev_routes_staging[b]))
+      return RR_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!host_qc[l] || !host_kc[l]) return RR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream, cs = (cudaStream_t)copy_stream;
+  cudaStream_t ds = d2h_stream ? (cudaStream_t)d2h_stream : cs;
+  const RRParams& p = L->p;
+  const size_t esz = p.dtype == RR_F32 ? 4 : 2;
+  const size_t qb = (size_t)p.P * p.n_q * p.d * esz, kb = (size_t)p.P * p.n_k * p.d * esz;
+  const size_t rb = (size_t)p.rows * p.k * 4;
+  for (int b = 0; b < 2; ++b) {
+    cudaEvent_t* evs[4] = {&L->ev_copied[b], &L->ev_consumed[b], &L->ev_snap[b], &L->ev_d2h[b]};
+    for (auto e : evs)
+      if (!*e) RR_CUDA(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+  }
+  // inputs of layer l -> staging set l%2 once layer l-2 has consumed it; issued one layer ahead
+  // so that the copy stream never queues an upload behind a download that waits for compute
+  auto upload = [&](int l) -> int {
+    const int b = l & 1;
+    if (l >= 2) RR_CUDA(cudaStreamWaitEvent(cs, L->ev_consumed[b], 0));
+    RR_CUDA(cudaMemcpyAsync(dev_qc_staging[b], host_qc[l], qb, cudaMemcpyHostToDevice, cs));
+    RR_CUDA(cudaMemcpyAsync(dev_kc_staging[b], host_kc[l], kb, cudaMemcpyHostToDevice, cs));
+    RR_CUDA(cudaEventRecord(L->ev_copied[b], cs));
+    return RR_OK;
+  };
+  if (n_layers > 0) { int rc = upload(0); if (rc != RR_OK) return rc; }
+  for (int l = 0; l < n_layers; ++l) {
+    const int b = l & 1;
+    RR_CUDA(cudaStreamWaitEvent(st, L->ev_copied[b], 0));
+    int rc = route_layer(L, dev_qc_staging[b], dev_kc_staging[b], first_layer + l,
+                         is_anchor[l] != 0, st);
+    if (rc != RR_OK) return rc;
+    RR_CUDA(cudaEventRecord(L->ev_consumed[b], st));
+    if (l + 1 < n_layers) { rc = upload(l + 1); if (rc != RR_OK) return rc; }
+    if (host_routes && host_routes[l]) {
+      // snapshot on the compute stream (device to device), copy out on the download stream
+      if (l >= 2) RR_CUDA(cudaStreamWaitEvent(st, L->ev_d2h[b], 0));
+      RR_CUDA(cudaMemcpyAsync(dev_routes_staging[b], p.routes, rb, cudaMemcpyDeviceToDevice, st));
+      RR_CUDA(cudaEventRecord(L->ev_snap[b], st));
+      RR_CUDA(cudaStreamWaitEvent(ds, L->ev_snap[b], 0));
+      RR_CUDA(cudaMemcpyAsync(host_routes[l], dev_routes_staging[b], rb, cudaMemcpyDeviceToHost, ds));
+      RR_CUDA(cudaEventRecord(L->ev_d2h[b], ds));
+    }
+  }
   return RR_OK;
 }
 

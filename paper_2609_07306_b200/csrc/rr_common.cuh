@@ -42,6 +42,9 @@ struct rr_ledger {
   bool profiling = false;
   struct ProfRec { int kind; cudaEvent_t a, b; };
   std::vector<ProfRec> prof;
+  // events of the pipelined host-buffer path (created on first use)
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr},
+              ev_snap[2] = {nullptr, nullptr}, ev_d2h[2] = {nullptr, nullptr};
 };
 
 // ---- device helpers -------------------------------------------------------------------

@@ -77,6 +77,19 @@ class RouteLedger:
                               host_routes.data_ptr() if host_routes is not None else None,
                               self._stream())
 
+    def route_layers_host(self, host_qc, host_kc, is_anchor, first_layer, dev_qc, dev_kc,
+                          dev_routes, host_routes, copy_stream: "torch.cuda.Stream",
+                          d2h_stream: "torch.cuda.Stream | None" = None):
+        """Lists of tensors (host: one per layer; device: two staging buffers each)."""
+        B.rr_route_layers_host(
+            self.handle, [t.data_ptr() for t in host_qc], [t.data_ptr() for t in host_kc],
+            list(is_anchor), first_layer, [t.data_ptr() for t in dev_qc],
+            [t.data_ptr() for t in dev_kc],
+            [t.data_ptr() for t in dev_routes] if dev_routes is not None else None,
+            [t.data_ptr() for t in host_routes] if host_routes is not None else None,
+            self._stream(), copy_stream.cuda_stream,
+            d2h_stream.cuda_stream if d2h_stream is not None else 0)
+
     def status(self) -> int:
         return B.rr_ledger_status(self.handle, self._stream())
 

@@ -168,6 +168,32 @@ def test_host_buffer_entry_point():
     led.close(); ref.close()
 
 
+def test_pipelined_host_layers_entry_point():
+    """rr_route_layers_host (copies overlapped on a second stream) returns, for every layer,
+    exactly the routes of the device-buffer calls."""
+    w = W.moderate().replace(heads=2)
+    L = 6
+    q, k = W.generate(w, layers=L)
+    led = RouteLedger(config_from_workload(w))
+    ref = RouteLedger(config_from_workload(w))
+    hq = [torch.from_numpy(q[l].view(np.int16)).pin_memory() for l in range(L)]
+    hk = [torch.from_numpy(k[l].view(np.int16)).pin_memory() for l in range(L)]
+    dq = [torch.empty_like(hq[0], device="cuda") for _ in range(2)]
+    dk = [torch.empty_like(hk[0], device="cuda") for _ in range(2)]
+    dr = [torch.empty(w.rows, w.k, dtype=torch.int32, device="cuda") for _ in range(2)]
+    outs = [torch.empty(w.rows, w.k, dtype=torch.int32).pin_memory() for _ in range(L)]
+    cs = torch.cuda.Stream()
+    anchors = [l % 3 == 0 for l in range(L)]
+    led.route_layers_host(hq, hk, anchors, 0, dq, dk, dr, outs, cs, torch.cuda.Stream())
+    torch.cuda.synchronize()
+    for l in range(L):
+        (ref.route_anchor if anchors[l] else ref.route_relay)(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        assert torch.equal(outs[l], ref.routes.cpu()), f"layer {l}"
+    assert led.counters_dict() == ref.counters_dict()
+    led.close(); ref.close()
+
+
 def test_token_ranges():
     w = W.moderate().replace(heads=2, chunk_tokens=64)
     q, k = W.generate(w, layers=2)
