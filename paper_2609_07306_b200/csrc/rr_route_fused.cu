@@ -403,7 +403,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       clear_bins(s);
     }
   }
-  bool usable = active && st.smax > st.smin && st.map_scale > 0.f && st.map_scale < 1e37f;
+  const bool usable = active && st.smax > st.smin && st.map_scale > 0.f && st.map_scale < 1e37f;
   const int from = usable ? st.binned : 0, to = usable ? n : 0;
   const int nw_new = warp_max(to - from);
   const float mlo = st.map_lo, msc = st.map_scale;
@@ -420,96 +420,47 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       aux_st(a, aux_ld(a) + (in ? 1u : 0u));
     }
   }
-  // (2) bin of rank keep, drop what lies below it.
-  // FINAL: rank keep and rank kk are located together, and instead of narrowing on the coarse
-  // bins a second, FINE histogram is laid over the coarse bins [b_keep, b_kk] (about one entry
-  // per fine bin), so that both ranks can almost always be finished without further levels.
+  // (2) bin of rank keep (and of rank kk), drop what lies below the former
   BinInfo bc, bk;
   int bsel, bsel_k = 0;
   scan_bins(s, keep, bsel, bc.cnt, bc.above);
   if (FINAL) scan_bins(s, kk, bsel_k, bk.cnt, bk.above);
   bc.reset(); bk.reset();
-  bool fine = false;
-  int rank_c = keep, rank_k = kk;                    // ranks inside what is left to search
-  if (FINAL) {
-    fine = usable && bsel >= 1 && bsel_k <= NB - 2 && bsel <= bsel_k;
-    usable = fine;                                    // others: search the whole buffer below
-    const int nd = fine ? n : 0;
-    const int nw = warp_max(nd);
-    const float flo = (float)bsel, fhi = (float)(bsel_k + 1), fs = (float)NB / (fhi - flo);
-    const int above_range = bk.above;                 // entries in coarse bins above b_kk
-    clear_bins_if(fine, s);
-    for (int e0 = 0; e0 < nw; e0 += BATCH) {
-      float v[BATCH];
+  const int nd = usable ? n : 0;
+  const int nw = warp_max(nd);
+  uint32_t waddr = s.buf;
+  // bin >= bsel  <=>  (v - lo) * scale >= bsel for bsel >= 1; bin 0 also holds what lies below lo
+  const float tb = bsel == 0 ? __int_as_float(0xff800000) : (float)bsel;
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH]; uint32_t id[BATCH];
 #pragma unroll
-      for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH);
+    for (int j = 0; j < BATCH; ++j)
+      ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
 #pragma unroll
-      for (int j = 0; j < BATCH; ++j) {
-        const float t = (v[j] - mlo) * msc;
-        const bool in = (e0 + j < nd) & (t >= flo) & (t < fhi);
-        const int f = max(0, min(NB - 1, __float2int_rz((t - flo) * fs)));
-        const uint32_t a = s.aux + f * AUX_PITCH;
-        aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+    for (int j = 0; j < BATCH; ++j) {
+      const float t = (v[j] - mlo) * msc;
+      const bool live = e0 + j < nd;
+      const bool keep_it = live & (t >= tb);
+      if (FINAL) {
+        const int b = max(0, min(NB - 1, __float2int_rz(t)));
+        bc.track(live & (b == bsel), v[j]);
+        bk.track(live & (b == bsel_k), v[j]);
+      } else {
+        bc.mn1 = fminf(bc.mn1, keep_it ? v[j] : bc.mn1);      // smallest survivor
       }
+      st_entry_if(keep_it, waddr, v[j], id[j]);
+      waddr += keep_it ? ENTRY_PITCH : 0u;
     }
-    int fsel, fsel_k;
-    scan_bins(s, keep - above_range, fsel, bc.cnt, bc.above);
-    scan_bins(s, kk - above_range, fsel_k, bk.cnt, bk.above);
-    uint32_t waddr = s.buf;
-    for (int e0 = 0; e0 < nw; e0 += BATCH) {
-      float v[BATCH]; uint32_t id[BATCH];
-#pragma unroll
-      for (int j = 0; j < BATCH; ++j)
-        ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
-#pragma unroll
-      for (int j = 0; j < BATCH; ++j) {
-        const float t = (v[j] - mlo) * msc;
-        const bool live = e0 + j < nd;
-        const bool in = live & (t >= flo) & (t < fhi);
-        const int f = max(0, min(NB - 1, __float2int_rz((t - flo) * fs)));
-        const bool keep_it = live & ((t >= fhi) | (in & (f >= fsel)));
-        bc.track(in & (f == fsel), v[j]);
-        bk.track(in & (f == fsel_k), v[j]);
-        st_entry_if(keep_it, waddr, v[j], id[j]);
-        waddr += keep_it ? ENTRY_PITCH : 0u;
-      }
-    }
-    if (fine) {
-      n = (int)((waddr - s.buf) / ENTRY_PITCH);
-      st.blo = bc.mn1;
-      rank_c = keep - above_range - bc.above;         // rank inside fine bin fsel
-      rank_k = kk - above_range - bk.above;           // rank inside fine bin fsel_k
-    }
-  } else {
-    const int nd = usable ? n : 0;
-    const int nw = warp_max(nd);
-    uint32_t waddr = s.buf;
-    // bin >= bsel <=> (v - lo) * scale >= bsel for bsel >= 1; bin 0 also holds what lies below lo
-    const float tb = bsel == 0 ? __int_as_float(0xff800000) : (float)bsel;
-    for (int e0 = 0; e0 < nw; e0 += BATCH) {
-      float v[BATCH]; uint32_t id[BATCH];
-#pragma unroll
-      for (int j = 0; j < BATCH; ++j)
-        ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
-#pragma unroll
-      for (int j = 0; j < BATCH; ++j) {
-        const float t = (v[j] - mlo) * msc;
-        const bool keep_it = (e0 + j < nd) & (t >= tb);
-        bc.mn1 = fminf(bc.mn1, keep_it ? v[j] : bc.mn1);        // smallest survivor
-        st_entry_if(keep_it, waddr, v[j], id[j]);
-        waddr += keep_it ? ENTRY_PITCH : 0u;
-      }
-    }
-    if (usable) {
-      n = (int)((waddr - s.buf) / ENTRY_PITCH);
-      st.binned = n;
-      st.blo = bc.mn1; st.tau = bc.mn1;  // >= keep seen scores reach mn1: a valid threshold
-    }
+  }
+  if (usable) {
+    n = (int)((waddr - s.buf) / ENTRY_PITCH);
+    st.binned = n;
+    st.blo = bc.mn1; st.tau = bc.mn1;  // >= keep seen scores reach mn1: a valid threshold
   }
   // (3) crowded bin, unusable range, or the final exact cut: finish inside b*
   const bool more = active && (!usable || n > fit_limit);
   float s_T = 0.f; int need = 0;
-  const bool direct = FINAL && more && usable && bc.resolve(rank_c, s_T, need);
+  const bool direct = FINAL && more && usable && bc.resolve(keep - bc.above, s_T, need);
   const bool zoom = more && !direct;
 #ifdef RR_PHASE_TIMING
   if (!FINAL) {       // ballots by the whole warp first; only then the lane-0 counters
@@ -525,7 +476,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     // FINAL and usable: everything left of interest is inside bin b* = [mn1, mx1] and `above`
     // entries outrank it; otherwise the whole (already reduced) buffer is searched
     const bool inbin = FINAL && usable;
-    select_rank(s, zoom, n, inbin ? rank_c : keep, true, fit_limit,
+    select_rank(s, zoom, n, inbin ? keep - bc.above : keep, true, fit_limit,
                 inbin ? bc.mn1 : (usable ? bc.mn1 : fminf(st.blo, st.smin)),
                 inbin ? bc.mx1 : st.smax, zs, zn, zexact);
     if (zoom) {
@@ -555,11 +506,11 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   if (FINAL) {
     const bool split = active && n > kk;
     float ks = 0.f; int kn = 0;
-    const bool kdirect = split && usable && bk.resolve(rank_k, ks, kn);
+    const bool kdirect = split && usable && bk.resolve(kk - bk.above, ks, kn);
     const bool kzoom = split && !kdirect;
     if (__any_sync(FULL, kzoom)) {
       float zs; int zn; bool zexact; int n_ = n;
-      select_rank(s, kzoom, n_, usable ? rank_k : kk, false, -1,
+      select_rank(s, kzoom, n_, usable ? kk - bk.above : kk, false, -1,
                   usable ? bk.mn1 : fminf(st.blo, st.smin), usable ? bk.mx1 : st.smax, zs, zn,
                   zexact);
       if (kzoom) { ks = zs; kn = zn; }
