@@ -6,19 +6,19 @@
 // compacted refresh list at a relay, Section 4.2) and walks the key chunks in tiles of 64,
 // stopping at the last chunk any of its rows may select.
 //   warp 0   : TMA producer (Kc tiles, 128-byte swizzle, 2-stage ring, no multicast)
-//   warp 1   : one thread issues tcgen05.mma (M=128, N=64, K=16) into a double-buffered TMEM
-//              accumulator
+//   warp 1   : one thread issues tcgen05.mma (M=128, N=64, K=16) into a ring of 4 TMEM
+//              accumulators
 //   warps 2-5: selection, ONE THREAD PER QUERY ROW (tcgen05.ld 32x32b hands each thread 32
 //              consecutive scores of its own row).  Each thread streams its row through a
-//              threshold filter into a private candidate buffer in shared memory
-//              (order-preserving 32-bit keys + chunk ids, laid out [slot][thread] so that
-//              accesses are bank-conflict free).  When a buffer nears its capacity the warp
-//              re-tightens: a 32-bin histogram over the buffer's key range finds the bin that
-//              holds the KEEP-th largest key (KEEP = k + max(m,1)), the threshold moves to that
-//              bin's lower edge and the buffer is compacted in place (stable, so entries stay
-//              in ascending chunk id).  After the last tile an exact multi-level histogram
-//              select (5 key bits per level) fixes rank KEEP and rank k; ties are resolved
-//              towards the smaller chunk id by buffer order.  The result is exact.
+//              threshold filter into a private candidate buffer in shared memory ({score,
+//              chunk id} entries laid out [slot][thread]: bank-conflict free).  When a buffer
+//              nears its capacity the warp re-tightens with a persistent 32-bin histogram of
+//              the buffered scores: the bin holding rank KEEP = k + max(m,1) is found, entries
+//              below it are dropped in place (stable, so entries stay in ascending chunk id)
+//              and the threshold moves to the smallest survivor.  After the last tile the cut
+//              at rank KEEP and the split at rank k are made exact inside their bins (directly
+//              for bins of up to 4 entries, else by zoom levels; a key-space radix level is
+//              the fallback for ranges too narrow to scale).  Ties go to the smaller chunk id.
 // Random sentinels are drawn by the same thread with the counter-based generator, using a
 // per-row bitmap of excluded chunks in shared memory.  Every mbarrier wait is bounded.
 #include "rr_common.cuh"
@@ -815,11 +815,21 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           if (pool > p.r) {
             const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
             const int limit = 64 * p.r;
-            for (int t = 0; t < limit && taken < p.r; ++t) {
-              const int j = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)t), (uint32_t)v);
-              const uint32_t wa = bm(j >> 5);
-              const uint32_t w = aux_ld(wa), bit = 1u << (j & 31);
-              if (!(w & bit)) { aux_st(wa, w | bit); rnd[taken++] = j; }
+            // four draws are generated at a time (independent 64-bit mixes overlap); they are
+            // still accepted strictly in draw order
+            for (int t0 = 0; t0 < limit && taken < p.r; t0 += 4) {
+              int j4[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                j4[i] = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)(t0 + i)), (uint32_t)v);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                if (t0 + i < limit && taken < p.r) {
+                  const uint32_t wa = bm(j4[i] >> 5);
+                  const uint32_t w = aux_ld(wa), bit = 1u << (j4[i] & 31);
+                  if (!(w & bit)) { aux_st(wa, w | bit); rnd[taken++] = j4[i]; }
+                }
+              }
             }
           }
           for (int j = 0; j < v && taken < p.r; ++j)
