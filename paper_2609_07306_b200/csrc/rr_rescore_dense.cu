@@ -3,14 +3,16 @@
 // The gathered kernel (rr_rescore.cu) fetches c Kc rows per query row and multiplies them on
 // the FP32 ALUs: no operand is reused, so it moves c*d*2 bytes per row through L2 and is an
 // order of magnitude slower on this machine than computing the whole score strip with
-// tcgen05.mma.  This variant does the latter: the same tile pipeline as the fused routing
-// kernel produces S[128 rows, 64 chunks] tiles in TMEM, and each row's thread picks out the
-// scores of its own candidates:
-//   * at start the thread turns its ledger row into three per-row bitmaps in shared memory
-//     (route, near-miss, all sentinels);
-//   * per tile it reads its 64 scores from TMEM and takes masked minima / maxima under the
-//     tile's bitmap words: alpha = min over route bits, beta = max over sentinel bits,
-//     floor = min over route and near-miss bits (the refresh's warm-start threshold).
+// tcgen05.mma.  This variant does the latter: the same kind of tile pipeline as the fused
+// routing kernel produces S[128 rows, 32 chunks] tiles in TMEM, and the threads of a row pick
+// out the scores of the row's candidates:
+//   * at start each warp turns ledger rows into per-row bitmaps in shared memory (two planes
+//     encoding route / near-miss / random sentinel), reading the ids with coalesced loads and
+//     setting bits with shared-memory OR reductions;
+//   * per tile a thread reads its share of the row's scores from TMEM and takes masked minima /
+//     maxima under the tile's bitmap words: alpha = min over route bits, beta = max over
+//     sentinel bits, floor = min over route and near-miss bits (the refresh's warm-start
+//     threshold).
 // Scores are bit-identical to the ones the fused routing kernel computes (same instruction
 // sequence on the same operands), so the floor needs no safety margin.
 // Outputs are those of the gathered kernel: flags, alpha, beta, tau, per-tile flagged counts,
@@ -23,16 +25,40 @@ using namespace sm100;
 namespace {
 
 // 32-chunk tiles keep a CTA under half an SM's shared memory: two CTAs per SM overlap one's
-// set-up and bitmap build with the other's tile loop.
-constexpr int BN = 32, B_STAGES = 3, ACC_STAGES = 4, NT = 192;
+// set-up and bitmap build with the other's tile loop.  Two threads share a query row (each
+// takes 16 of a tile's 32 columns): the per-tile work is a chain of dependent ALU-pipe
+// instructions, so twice the warps hide twice the latency.
+constexpr int BN = 32, B_STAGES = 3, ACC_STAGES = 4;
+constexpr int TPR = 2, COLS = BN / TPR;             // threads per row, columns per thread
+constexpr int NCONS = tcpipe::BM * TPR, NT = 64 + NCONS;
+constexpr int ROWS_PER_WARP = 32 / TPR;             // ledger rows a warp turns into bitmaps
 constexpr unsigned FULL = 0xFFFFFFFFu;
-constexpr uint32_t PITCH = tcpipe::BM * 4;          // one 32-bit word per row thread
+constexpr uint32_t PITCH = tcpipe::BM * 4;          // debug score column: one word per row
 
 __device__ __forceinline__ uint32_t lds(uint32_t a) {
   uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v;
 }
 __device__ __forceinline__ void sts(uint32_t a, uint32_t v) {
   asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+// no memory clobber: the loads of the next rows' ids may move across it
+__device__ __forceinline__ void red_or(uint32_t a, uint32_t v) {
+  asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(a), "r"(v));
+}
+__device__ __forceinline__ void sts_zero16(uint32_t a) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void consumers_sync() {            // the NCONS consumer threads only
+  asm volatile("bar.sync 1, %0;" ::"n"(NCONS) : "memory");
+}
+// acc = min(acc, s) / max(acc, s) if (word & bit): a predicate and a predicated instruction
+__device__ __forceinline__ void min_if(float& acc, float s, uint32_t word, uint32_t bit) {
+  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %2, %3;\n\tsetp.ne.u32 p, t, 0;\n\t"
+      "@p min.f32 %0, %0, %1;\n\t}" : "+f"(acc) : "f"(s), "r"(word), "r"(bit));
+}
+__device__ __forceinline__ void max_if(float& acc, float s, uint32_t word, uint32_t bit) {
+  asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %2, %3;\n\tsetp.ne.u32 p, t, 0;\n\t"
+      "@p max.f32 %0, %0, %1;\n\t}" : "+f"(acc) : "f"(s), "r"(word), "r"(bit));
 }
 
 #ifdef RR_PHASE_TIMING
@@ -44,18 +70,26 @@ __device__ unsigned long long g_rd_phase[8];
 #define RD_LAP(i) do {} while (0)
 #endif
 
+// Per-row bitmaps: row r owns `pitch` = 2*words + 1 consecutive words (odd, so that the 32 rows
+// of a warp fall into 32 different banks when each thread reads word t of its own row, and the
+// words of one row fall into different banks when a warp builds that row together).
+// Two planes encode the three candidate classes of a chunk:
+//   plane A | plane B :  route = 1|0,  near-miss = 0|1,  random sentinel = 1|1.
 template <int D>
 __global__ void __launch_bounds__(NT, 2)
-rescore_dense_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
+rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int words) {
-  using P = tcpipe::Pipe<D, BN, B_STAGES, ACC_STAGES>;
+  using P = tcpipe::Pipe<D, BN, B_STAGES, ACC_STAGES, NCONS>;
   extern __shared__ uint8_t smem_raw[];
   P pipe;
   pipe.carve(smem_raw);
-  // extra: 3 counters, [3*words][128] bitmap words, (debug only) [BN][128] score column
+  // extra: 3 counters, [128][pitch] bitmap words, [3][128] partial results of the second
+  // thread of each row, (debug only) [BN][128] score column
   unsigned long long* s_cnt = (unsigned long long*)pipe.extra;
+  const uint32_t pitch = 2u * words + 1u;
   const uint32_t bm_base = smem_u32(pipe.extra) + 64u;
-  const uint32_t sc_base = bm_base + 3u * words * PITCH;
+  const uint32_t xch_base = (bm_base + tcpipe::BM * pitch * 4u + 15u) & ~15u;
+  const uint32_t sc_base = xch_base + 3u * PITCH;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tiles_m = p.tiles_per_problem;
@@ -63,82 +97,104 @@ rescore_dense_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   const int tile_id = prob * tiles_m + tm;
   if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; }
   RD_T0();
-  pipe.setup(p, qc, &tmap_k, nullptr, prob, tm, 0, p.n_q, NT);
+  pipe.setup(p, nullptr, &tmap_k, nullptr, prob, tm, 0, p.n_q, NT, &tmap_q);
   const int n_tiles = pipe.num_tiles(p);
 
   if (warp == 0) {
-    if (lane == 0) pipe.producer(&tmap_k, prob, n_tiles);
+    if (lane == 0) pipe.producer(&tmap_k, prob, n_tiles, &tmap_q, tm);
   } else if (warp == 1) {
-    if (lane == 0) pipe.mma_issuer(n_tiles);
+    if (lane == 0) pipe.mma_issuer(n_tiles, true);
   } else {
-    const int quarter = warp & 3;
+    // a warp may only read the TMEM lanes 32*(warp % 4) ...: warps 2-5 take the first COLS
+    // columns of their quarter's rows, warps 6-9 the rest
+    const int quarter = warp & 3, part = (warp - 2) >> 2;
     const int r = quarter * 32 + lane;
-    const int row = pipe.ctl->row[r];
-    const int g = pipe.ctl->slot[r];
+    const int row = tm * tcpipe::BM + r < p.n_q ? tm * tcpipe::BM + r : -1;   // rows are consecutive
+    const int g = prob * p.n_q + tm * tcpipe::BM + r;
     const int v = row >= 0 ? rr_valid_count(row, p.n_k, p.causal, p.causal_offset) : 0;
-    const uint32_t bR = bm_base + r * 4u, bN = bR + words * PITCH, bS = bN + words * PITCH;
+    const uint32_t bA = bm_base + r * pitch * 4u, bB = bA + words * 4u;
     const uint32_t col = sc_base + r * 4u;
     const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
 
     RD_LAP(0);
-    // ---- ledger row -> bitmaps ---------------------------------------------------------------
-    for (int w = 0; w < 3 * words; ++w) sts(bR + w * PITCH, 0u);
-    int n_valid = 0; bool bad = false;
-    if (row >= 0) {
-      const int32_t* route = p.routes + (size_t)g * p.k;
-      const int32_t* sent = p.sentinels + (size_t)g * p.sw;
-      // ids are fetched 16 at a time, all loads first: one L2 round trip per group, not per id
-      for (int s0 = 0; s0 < p.c; s0 += 16) {
-        int ids[16];
+    // ---- ledger rows -> bitmaps: each warp builds ROWS_PER_WARP rows, all lanes together ------
+    {
+      const int rb = quarter * 32 + part * ROWS_PER_WARP;          // first row of this warp's share
+      const uint32_t wbase = bm_base + (uint32_t)rb * pitch * 4u;  // 16-byte aligned stretch
+      for (uint32_t o = lane * 16u; o < (uint32_t)ROWS_PER_WARP * pitch * 4u; o += 512u)
+        sts_zero16(wbase + o);
+      __syncwarp();
+      RD_LAP(4);
+      int n_ok = 0; bool bad = false;
+      const int row_b = tm * tcpipe::BM + rb;
+      // lane L takes candidate slots L, L+32, ...: the ids of a row are read with coalesced
+      // loads, all rows in flight at once, and set with fire-and-forget shared-memory ORs
+      for (int s0 = 0; s0 < p.c; s0 += 32) {
+        const int s = s0 + lane;
+        const bool is_route = s < p.k, is_near = !is_route && s < p.k + p.m;
+        const int32_t* src = is_route ? p.routes + ((size_t)prob * p.n_q + row_b) * p.k + s
+                                      : p.sentinels + ((size_t)prob * p.n_q + row_b) * p.sw + (s - p.k);
+        const int stride = is_route ? p.k : p.sw;
+        int ids[ROWS_PER_WARP];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int s = s0 + j;
-          ids[j] = s < p.k ? __ldg(route + s) : (s < p.c ? __ldg(sent + (s - p.k)) : -1);
-        }
+        for (int j = 0; j < ROWS_PER_WARP; ++j)
+          ids[j] = (row_b + j < p.n_q && s < p.c) ? __ldg(src + (size_t)j * stride) : -1;
+        const uint32_t plane_a = is_near ? 0u : 1u, plane_b = is_route ? 0u : 1u;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int s = s0 + j, id = ids[j];
-          bad |= id >= v;
-          const bool ok = (id >= 0) & (id < v);
-          const uint32_t wi = ok ? (uint32_t)(id >> 5) : 0u, bit = ok ? 1u << (id & 31) : 0u;
-          const uint32_t a = (s < p.k ? bR : bS) + wi * PITCH;
-          sts(a, lds(a) | bit);
-          if (s >= p.k && s < p.k + p.m) { const uint32_t an = bN + wi * PITCH; sts(an, lds(an) | bit); }
-          n_valid += ok;
-          if (p.debug && s < p.c) p.cand_scores[(size_t)g * p.c + s] = __int_as_float(0x7fc00000);
+        for (int j = 0; j < ROWS_PER_WARP; ++j) {
+          const int vj = rr_valid_count(row_b + j, p.n_k, p.causal, p.causal_offset);
+          const int id = ids[j];
+          bad |= id >= vj;
+          if (id >= 0 && id < vj) {
+            const uint32_t a = wbase + ((uint32_t)j * pitch + (uint32_t)(id >> 5)) * 4u;
+            const uint32_t bit = 1u << (id & 31);
+            if (plane_a) red_or(a, bit);
+            if (plane_b) red_or(a + words * 4u, bit);
+            ++n_ok;
+          }
+          if (p.debug && row_b + j < p.n_q && s < p.c)
+            p.cand_scores[((size_t)prob * p.n_q + row_b + j) * p.c + s] = __int_as_float(0x7fc00000);
         }
       }
+      if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
+      n_ok = __reduce_add_sync(FULL, n_ok);
+      if (lane == 0) atomicAdd(&s_cnt[1], (unsigned long long)n_ok);
     }
-    if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
+    consumers_sync();                    // a row's bitmap is read by warps that did not build it
 
     float amin = pinf, bmax = ninf, nmin = pinf;      // nmin: weakest near-miss candidate
     bool alive = true;
+    const uint32_t sh = (uint32_t)part * COLS;
     RD_LAP(1);
     for (int t = 0; t < n_tiles; ++t) {
-      if (!pipe.consumer_wait(t)) { alive = false; break; }
+      // after a wait that gave up the remaining iterations only keep the barriers in step
+      if (alive) alive = pipe.consumer_wait(t);
       RD_LAP(2);
       static_assert(BN == 32, "a tile is one bitmap word");
-      const bool in = t < words;
-      const uint32_t wr = in ? lds(bR + t * PITCH) : 0u, wn = in ? lds(bN + t * PITCH) : 0u;
-      const uint32_t ws = in ? lds(bS + t * PITCH) : 0u;
-      if (__any_sync(FULL, (wr | ws) != 0u)) {
-        uint32_t a0[32];
-        tmem_ld_32x32(pipe.acc_addr(t, quarter), a0);
+      const bool in = alive && t < words;
+      const uint32_t wa = in ? lds(bA + t * 4u) >> sh : 0u, wb = in ? lds(bB + t * 4u) >> sh : 0u;
+      const uint32_t wr = wa & ~wb, wn = wb & ~wa, ws = wb;
+      const bool work = __any_sync(FULL, ((wa | wb) & ((1u << COLS) - 1u)) != 0u);
+      uint32_t a0[COLS];
+      if (work) {
+        tmem_ld_32x16(pipe.acc_addr(t, quarter) + sh, a0);
         // masked min / max straight from the registers: no loop over set bits (its trip
         // count and its dependent shared-memory reads made it several times slower)
 #pragma unroll
-        for (int q = 0; q < 32; ++q) {
+        for (int q = 0; q < COLS; ++q) {
           const float s0 = __uint_as_float(a0[q]);
-          const uint32_t bit = 1u << q;
-          amin = fminf(amin, (wr & bit) ? s0 : pinf);
-          bmax = fmaxf(bmax, (ws & bit) ? s0 : ninf);
-          nmin = fminf(nmin, (wn & bit) ? s0 : pinf);
+          min_if(amin, s0, wr, 1u << q);
+          max_if(bmax, s0, ws, 1u << q);
+          min_if(nmin, s0, wn, 1u << q);
         }
-        if (p.debug) {
+      }
+      if (p.debug) {                                         // tests: every candidate's score
+        if (work) {
 #pragma unroll
-          for (int q = 0; q < 32; ++q) sts(col + q * PITCH, a0[q]);
+          for (int q = 0; q < COLS; ++q) sts(col + (sh + q) * PITCH, a0[q]);
         }
-        if (p.debug && row >= 0) {                            // tests: every candidate's score
+        consumers_sync();
+        if (alive && part == 0 && row >= 0) {
           const int32_t* route = p.routes + (size_t)g * p.k;
           const int32_t* sent = p.sentinels + (size_t)g * p.sw;
           for (int s = 0; s < p.c; ++s) {
@@ -148,21 +204,38 @@ rescore_dense_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
               p.cand_scores[(size_t)g * p.c + s] = __uint_as_float(lds(col + (uint32_t)rel * PITCH));
           }
         }
+        consumers_sync();
       }
-      pipe.consumer_release(t);
+      if (alive) pipe.consumer_release(t);
       RD_LAP(3);
     }
 
-    if (alive && row >= 0) {
+    // ---- the second thread of each row hands its partial results to the first ---------------
+    if (part != 0) {
+      sts(xch_base + r * 4u, __float_as_uint(amin));
+      sts(xch_base + PITCH + r * 4u, __float_as_uint(bmax));
+      sts(xch_base + 2u * PITCH + r * 4u, __float_as_uint(nmin));
+    }
+    consumers_sync();
+    if (part == 0) {
+      amin = fminf(amin, __uint_as_float(lds(xch_base + r * 4u)));
+      bmax = fmaxf(bmax, __uint_as_float(lds(xch_base + PITCH + r * 4u)));
+      nmin = fminf(nmin, __uint_as_float(lds(xch_base + 2u * PITCH + r * 4u)));
+      const bool ok = alive && row >= 0;
       const bool has_sent = bmax > ninf;
-      const bool flag = has_sent && !(amin > bmax + p.gamma);
-      p.flags[g] = flag ? 1 : 0;
-      p.alpha[g] = amin;
-      p.beta[g] = bmax;
-      p.tau[g] = p.m > 0 ? fminf(amin, nmin) : ninf;    // floor of the k+m old candidates
-      atomicAdd(&s_cnt[0], (unsigned long long)flag);
-      atomicAdd(&s_cnt[1], (unsigned long long)n_valid);
-      if (flag) atomicAdd(&s_cnt[2], (unsigned long long)v);
+      const bool flag = ok && has_sent && !(amin > bmax + p.gamma);
+      if (ok) {
+        p.flags[g] = flag ? 1 : 0;
+        p.alpha[g] = amin;
+        p.beta[g] = bmax;
+        p.tau[g] = p.m > 0 ? fminf(amin, nmin) : ninf;    // floor of the k+m old candidates
+      }
+      const int n_flag = __popc(__ballot_sync(FULL, flag));
+      const int v_sum = __reduce_add_sync(FULL, flag ? v : 0);
+      if (lane == 0) {
+        atomicAdd(&s_cnt[0], (unsigned long long)n_flag);
+        atomicAdd(&s_cnt[2], (unsigned long long)v_sum);
+      }
     }
   }
 
@@ -177,9 +250,9 @@ rescore_dense_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 
 size_t smem_need(const RRParams& p, int& words) {
   words = (p.n_k + 31) / 32;
-  const size_t fixed = p.d == 128 ? tcpipe::Pipe<128, BN, B_STAGES, ACC_STAGES>::FIXED_BYTES
-                                  : tcpipe::Pipe<64, BN, B_STAGES, ACC_STAGES>::FIXED_BYTES;
-  return fixed + (size_t)(3 * words + (p.debug ? BN : 0)) * PITCH + 64;
+  const size_t fixed = p.d == 128 ? tcpipe::Pipe<128, BN, B_STAGES, ACC_STAGES, NCONS>::FIXED_BYTES
+                                  : tcpipe::Pipe<64, BN, B_STAGES, ACC_STAGES, NCONS>::FIXED_BYTES;
+  return fixed + (size_t)tcpipe::BM * (2 * words + 1) * 4 + 16 + (size_t)(3 + (p.debug ? BN : 0)) * PITCH + 64;
 }
 
 }  // namespace
@@ -202,8 +275,10 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
                                     cudaStream_t st) {
   int words;
   const size_t smem = smem_need(p, words);
-  CUtensorMap tmap;
+  CUtensorMap tmap, tmap_q;
   cudaError_t e = rr_encode_tmap_bf16_3d(&tmap, kc, p.d, p.n_k, p.P, BN);
+  if (e != cudaSuccess) return e;
+  e = rr_encode_tmap_bf16_3d(&tmap_q, qc, p.d, p.n_q, p.P, tcpipe::BM);
   if (e != cudaSuccess) return e;
   static bool attr_set = false;
   if (!attr_set) {
@@ -219,9 +294,9 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
   }
   const int grid = p.n_tiles;
   if (p.d == 128)
-    rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, words);
+    rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words);
   else
-    rescore_dense_kernel<64><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, words);
+    rescore_dense_kernel<64><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words);
   rr_count_launch();
   return cudaPeekAtLastError();
 }

@@ -568,12 +568,23 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   {
     constexpr int CPR = D / 8;
     const __nv_bfloat16* qbase = qc + (size_t)prob * p.n_q * D;
-    for (int ch = tid; ch < BM * CPR; ch += NT) {
-      const int r = ch / CPR, c16 = ch % CPR, h = c16 >> 3, cc = c16 & 7;
-      const int row = ctl->row[r];
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (row >= 0) v = __ldg(reinterpret_cast<const uint4*>(qbase + (size_t)row * D + c16 * 8));
-      *reinterpret_cast<uint4*>(sA + h * C::A_HALF + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+    // all of a thread's loads are issued before its first store: one memory round trip
+    constexpr int ITER = (BM * CPR + NT - 1) / NT;
+    uint4 vals[ITER];
+#pragma unroll
+    for (int i = 0; i < ITER; ++i) {
+      const int ch = tid + i * NT, r = ch / CPR, c16 = ch % CPR;
+      vals[i] = make_uint4(0, 0, 0, 0);
+      if (ch < BM * CPR) {
+        const int row = ctl->row[r];
+        if (row >= 0) vals[i] = __ldg(reinterpret_cast<const uint4*>(qbase + (size_t)row * D + c16 * 8));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < ITER; ++i) {
+      const int ch = tid + i * NT, r = ch / CPR, c16 = ch % CPR, h = c16 >> 3, cc = c16 & 7;
+      if (ch < BM * CPR)
+        *reinterpret_cast<uint4*>(sA + h * C::A_HALF + r * 128 + ((cc ^ (r & 7)) << 4)) = vals[i];
     }
     fence_proxy_async_smem();
   }

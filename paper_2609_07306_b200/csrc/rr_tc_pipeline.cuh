@@ -4,10 +4,12 @@
 //                    of B_STAGES shared-memory stages
 //   warp 1, lane 0 : issues tcgen05.mma (M=128, N=BN, K=16; d/16 steps per tile) into a ring of
 //                    ACC_STAGES TMEM accumulators of BN columns and commits to mbarriers
-//   consumers      : 128 threads, one per row; wait on acc_full[stage], read TMEM with
-//                    tcgen05.ld, then arrive on acc_empty[stage]
+//   consumers      : CONSUMERS threads (one or more per row); wait on acc_full[stage], read
+//                    TMEM with tcgen05.ld, then arrive on acc_empty[stage]
 // The Qc tile is gathered by all threads with 16-byte loads straight into the swizzled layout
-// the MMA descriptors expect (rows of a refresh list are not contiguous in memory).
+// the MMA descriptors expect (rows of a refresh list are not contiguous in memory); when the
+// rows are consecutive the caller may hand a tensor map of Qc instead, and the producer fetches
+// the tile with TMA while the consumers are already busy with their own set-up.
 // Every mbarrier wait is bounded: on expiry the abort flag is raised, every role leaves its
 // loop, the CTA frees its TMEM and reports RR_STATUS_TIMEOUT.
 #pragma once
@@ -20,7 +22,7 @@ using namespace sm100;
 
 constexpr int BM = 128;
 
-template <int D, int BN, int B_STAGES, int ACC_STAGES>
+template <int D, int BN, int B_STAGES, int ACC_STAGES, int CONSUMERS = BM>
 struct Pipe {
   static constexpr int KHALVES = D / 64, KSTEPS = D / 16;
   static constexpr int A_BYTES = BM * D * 2, B_BYTES = BN * D * 2;
@@ -31,6 +33,7 @@ struct Pipe {
 
   struct Ctl {
     uint64_t full[B_STAGES], empty[B_STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+    uint64_t a_full;                                      // Qc tile landed (TMA variant only)
     uint32_t tmem_base, abort_flag;
     int row[BM], slot[BM];
   };
@@ -47,9 +50,11 @@ struct Pipe {
 
   // Row table, barriers, TMEM allocation, Qc tile.  Call with all threads; ends in a
   // __syncthreads().  rows come from row_list[seg_lo + tm*BM ...) (relay) or are consecutive.
+  // tmap_q != nullptr (consecutive rows only): the Qc tile is left to producer().
   __device__ __forceinline__ void setup(const RRParams& p, const __nv_bfloat16* qc,
                                         const CUtensorMap* tmap_k, const int32_t* row_list,
-                                        int prob, int tm, int seg_lo, int seg_hi, int nthreads) {
+                                        int prob, int tm, int seg_lo, int seg_hi, int nthreads,
+                                        const CUtensorMap* tmap_q = nullptr) {
     const int tid = threadIdx.x, warp = tid >> 5;
     if (tid < BM) {
       const int local = tm * BM + tid;
@@ -64,12 +69,20 @@ struct Pipe {
     }
     if (tid == 0) {
       for (int s = 0; s < B_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-      for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(&ctl->acc_full[s], 1); mbar_init(&ctl->acc_empty[s], BM); }
+      for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(&ctl->acc_full[s], 1); mbar_init(&ctl->acc_empty[s], CONSUMERS); }
+      mbar_init(&ctl->a_full, 1);
       ctl->abort_flag = 0;
       mbar_fence_init();
       tma_prefetch_desc(tmap_k);
+      if (tmap_q) tma_prefetch_desc(tmap_q);
     }
     if (warp == 0) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+    if (tmap_q) {
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      return;
+    }
     __syncthreads();
     constexpr int CPR = D / 8;                            // 16-byte chunks per row
     const __nv_bfloat16* qbase = qc + (size_t)prob * p.n_q * D;
@@ -94,8 +107,15 @@ struct Pipe {
     return (vmax + BN - 1) / BN;
   }
 
-  __device__ __forceinline__ void producer(const CUtensorMap* tmap_k, int prob, int n_tiles) {
+  __device__ __forceinline__ void producer(const CUtensorMap* tmap_k, int prob, int n_tiles,
+                                           const CUtensorMap* tmap_q = nullptr, int tm = 0) {
     volatile uint32_t* abort_flag = &ctl->abort_flag;
+    if (tmap_q) {                                         // rows past n_q are zero-filled
+      mbar_expect_tx(&ctl->a_full, A_BYTES);
+#pragma unroll
+      for (int h = 0; h < KHALVES; ++h)
+        tma_load_3d(sA + h * A_HALF, tmap_q, h * 64, tm * BM, prob, &ctl->a_full);
+    }
     int issued = 0;
     for (int t = 0; t < n_tiles; ++t) {
       const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
@@ -111,10 +131,13 @@ struct Pipe {
       const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
       for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->full[s], ph); ++it) __nanosleep(64);
     }
+    if (tmap_q)
+      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->a_full, 0); ++it) __nanosleep(64);
   }
 
-  __device__ __forceinline__ void mma_issuer(int n_tiles) {
+  __device__ __forceinline__ void mma_issuer(int n_tiles, bool q_by_tma = false) {
     volatile uint32_t* abort_flag = &ctl->abort_flag;
+    if (q_by_tma && !mbar_wait(&ctl->a_full, 0, abort_flag)) return;
     constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
     const uint32_t a_addr = smem_u32(sA);
     const uint32_t tmem_base = ctl->tmem_base;
