@@ -106,12 +106,32 @@ def long_ctx() -> RouteWorkload:
                          chunk_tokens=64)
 
 
+def low_drift() -> RouteWorkload:
+    """The headline shape in the regime the method is built for: slow drift, few flagged rows."""
+    return RouteWorkload("low_drift", 8, 32, 1024, 1024, 128, 32, 16, 16, layers=32,
+                         anchor_every=8, dtype=DTYPE_BF16, centroids=64, rho=0.005, causal=True)
+
+
+def ablation(m: int = 12, r: int = 12) -> RouteWorkload:
+    """Shape of the sentinel-ablation table (Section 5.2): 256 x 256 chunks, top-12 routes,
+    24 layers with a single anchor at layer 0; (m, r) = (0, 0) is the fixed-stride baseline."""
+    return RouteWorkload(f"ablation_m{m}_r{r}", 8, 32, 256, 256, 128, 12, m, r, layers=24,
+                         anchor_every=24, dtype=DTYPE_BF16, centroids=32, rho=0.003, causal=False)
+
+
 PRESETS = {
     "tiny": tiny,
     "moderate": moderate,
     "sweep": sweep,
     "high_drift": high_drift,
     "long_ctx": long_ctx,
+    "low_drift": low_drift,
+    "ablation_m0_r12": lambda: ablation(0, 12),
+    "ablation_m12_r12": lambda: ablation(12, 12),
+    "ablation_m24_r12": lambda: ablation(24, 12),
+    "ablation_m48_r12": lambda: ablation(48, 12),
+    "ablation_m12_r0": lambda: ablation(12, 0),
+    "fixed_stride": lambda: ablation(0, 0),
 }
 
 

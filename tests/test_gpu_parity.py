@@ -231,3 +231,39 @@ def test_free_running_summary_matches_oracle():
     assert abs(rer - summ.rerouted_fraction) < 2e-3
     assert abs(pairs - summ.score_pair_fraction) < 2e-3
     led.close()
+
+
+@pytest.mark.parametrize("m,r", [(0, 12), (12, 12), (48, 12), (12, 0), (0, 0)])
+def test_sentinel_ablation_shapes(m, r):
+    """The (m, r) grid of the sentinel-ablation table (Section 5.2), including random-only,
+    near-miss-only and the fixed-stride baseline m = r = 0 (nothing can challenge a route)."""
+    w = W.ablation(m, r).replace(batch=1, heads=3, layers=5)
+    for two_pass, gathered in ((False, False), (False, True), (True, True)):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
+        _report(rep)
+        parity.assert_clean(rep)
+
+
+def test_fixed_stride_never_flags_and_low_drift_flags_few():
+    """Free-running: with m = r = 0 only the anchor layer routes (rerouted fraction 1/L; the
+    pairs are the anchor's plus k per relay row); at low drift the flagged fraction stays far below the high-drift regime's."""
+    def run(w):
+        q, k = W.generate(w)
+        led = RouteLedger(config_from_workload(w))
+        for l in range(w.layers):
+            fn = led.route_anchor if w.is_anchor(l) else led.route_relay
+            fn(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        c = led.counters_dict()
+        led.close()
+        return O.fractions_from_counters(c)
+    w = W.ablation(0, 0).replace(batch=1, heads=4, layers=6)
+    rer, flg, pairs = run(w)
+    assert flg == 0.0 and abs(rer - 1 / 6) < 1e-12
+    assert abs(pairs - (1 / 6 + (5 / 6) * 12 / 256)) < 1e-12
+    w = W.low_drift().replace(batch=1, heads=2, layers=4)
+    rer, flg, pairs = run(w)
+    w_hi = W.high_drift().replace(batch=1, heads=2, layers=4, redraw_every=0)
+    _, flg_hi, _ = run(w_hi)
+    print(f"flagged fraction: low drift {flg:.3f}, high drift {flg_hi:.3f}")
+    assert flg < 0.5 * flg_hi
