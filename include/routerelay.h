@@ -80,12 +80,25 @@ typedef struct rr_config {
                               + warp-level TopK) even where the fused kernel applies;
                               bit 2: rescore candidates with the gathered FP32 kernel even
                               where the tensor-core strip kernel applies                  */
+  /* Optional policies either side of the trigger; all zero = the plain method.             */
+  int32_t global_sentinels;/* mandatory global candidates (Section 3.1, item 3): bit 0 = the
+                              sink chunk 0, bit 1 = the most recent chunk the row may select.
+                              Each adds one slot after the random sentinels; a slot stays -1
+                              if its chunk is in the route or among the near-miss sentinels;
+                              the random sentinels are drawn from what is left              */
+  int32_t min_reuse;       /* hysteresis (Section 3.2): a row fully routed fewer than this
+                              many layers ago is reused without the test (the paper: 1)     */
+  int32_t h_max;           /* forced anchors (Section 3.2), per row: >0 = a row whose route
+                              is h_max or more layers old is re-routed whatever Eq. 5 says  */
+  float   gamma_boost;     /* hysteresis: added to gamma for rows whose margin (Section 3.3)
+                              recorded at their last routing is below margin_recover        */
+  float   margin_recover;
 } rr_config;
 
 /* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */
 typedef struct rr_views {
   int32_t* routes;          /* [rows, k]     selected chunk ids                             */
-  int32_t* sentinels;       /* [rows, m+r]   near-miss (first m) then random (last r)       */
+  int32_t* sentinels;       /* [rows, m+r+g] near-miss (m), random (r), then g mandatory global slots */
   int32_t* ages;            /* [rows]        layers since the row was last fully routed; -1 after reset */
   float*   kth_score;       /* [rows]        weakest selected score when last routed        */
   float*   margin;          /* [rows]        Section 3.3 margin when last routed (+inf if nothing is unselected) */
@@ -96,7 +109,7 @@ typedef struct rr_views {
   int32_t* refresh_count;   /* [1]           how many (= rho_l * rows)                      */
   int32_t* problem_offsets; /* [P+1]         exclusive scan of per-problem flagged counts   */
   int32_t* token_ranges;    /* [rows, k, 2]  [start,end) per route slot, ascending chunk id; NULL if chunk_tokens==0 */
-  float*   cand_scores;     /* [rows, k+m+r] candidate scores of the last relay; NULL unless debug_outputs */
+  float*   cand_scores;     /* [rows, k+m+r+g] candidate scores of the last relay; NULL unless debug_outputs */
   uint64_t* counters;       /* [RR_NUM_COUNTERS] cumulative since reset, see below          */
   uint32_t* status;         /* [1]           RR_STATUS_* bits                               */
 } rr_views;

@@ -17,7 +17,11 @@ current layer), so the oracle follows the algorithm step by step:
           sentinels rebuilt;
 * Sec 4.1 unstable row ids are compacted in ascending order; stable rows keep route and
           sentinels and their age advances; rebuilt rows get age 0;
-* Sec 3.3 anchor margin Delta = min selected - max unselected.
+* Sec 3.3 anchor margin Delta = min selected - max unselected;
+* Sec 3.1 item 3 / Sec 3.2 (optional policies, off by default): mandatory global sentinels
+          (sink chunk, most recent chunk), a minimum reuse horizon and a larger guard margin
+          for rows whose recorded margin is small (hysteresis), forced re-routing of rows
+          whose route is h_max layers old (forced anchors, per row).
 
 Readings of points the paper leaves open are listed in the design notes of the
 repository; the ones that matter here: ties break towards the smaller chunk index;
@@ -115,10 +119,25 @@ class OracleParams:
     causal: bool = False
     causal_offset: int = 0
     seed: int = 0
+    # policies either side of the trigger (Sec 3.1 item 3, Sec 3.2 "Hysteresis", "Forced anchors")
+    global_sentinels: int = 0     # bit 0: sink chunk 0, bit 1: most recent valid chunk
+    min_reuse: int = 0            # a row routed fewer than this many layers ago is not tested
+    gamma_boost: float = 0.0      # added to gamma while the row's recorded margin < margin_recover
+    margin_recover: float = 0.0
+    h_max: int = 0                # >0: a row last routed h_max or more layers ago is re-routed
+
+    @property
+    def n_global(self) -> int:
+        return (self.global_sentinels & 1) + ((self.global_sentinels >> 1) & 1)
+
+    @property
+    def sw(self) -> int:
+        """Width of a sentinel row: near-miss, random, then mandatory global slots."""
+        return self.m + self.r + self.n_global
 
     @property
     def c(self) -> int:
-        return self.k + self.m + self.r
+        return self.k + self.sw
 
     def valid_counts(self) -> np.ndarray:
         """v_i: how many key chunks query row i may select."""
@@ -133,7 +152,7 @@ class Ledger:
     """Route-maintenance state (Sec 4.1): routes, sentinels (near-miss then random), ages,
     plus the k-th score and margin recorded when each row was last routed."""
     routes: np.ndarray      # [rows, k] int32, -1 = empty slot
-    sentinels: np.ndarray   # [rows, m+r] int32
+    sentinels: np.ndarray   # [rows, m+r+globals] int32
     ages: np.ndarray        # [rows] int32, -1 = never routed
     kth: np.ndarray         # [rows] float64
     margin: np.ndarray      # [rows] float64
@@ -141,7 +160,7 @@ class Ledger:
     @staticmethod
     def empty(rows: int, p: OracleParams) -> "Ledger":
         return Ledger(np.full((rows, p.k), -1, np.int32),
-                      np.full((rows, p.m + p.r), -1, np.int32),
+                      np.full((rows, p.sw), -1, np.int32),
                       np.full(rows, -1, np.int32),
                       np.zeros(rows, np.float64), np.zeros(rows, np.float64))
 
@@ -180,15 +199,27 @@ def full_route(s_row: np.ndarray, v: int, k: int) -> np.ndarray:
 def route_row(s_row: np.ndarray, v: int, p: OracleParams, g: int, layer: int):
     """Full routing of one row plus sentinel construction (Sec 3.1) and margin (Sec 3.3).
 
-    Returns (route[k], sentinels[m+r], kth_score, margin) with -1 padding."""
+    Sentinel row: m near-miss slots, r random slots, then one slot per mandatory global
+    candidate (sink = chunk 0, recent = the last chunk the row may select).  A global
+    candidate that is already in the route or among the near-miss sentinels (or equals an
+    earlier global one) leaves its slot empty; the random sentinels are drawn from what is
+    left after route, near-miss and global candidates.
+
+    Returns (route[k], sentinels[sw], kth_score, margin) with -1 padding."""
     order = rank_order(s_row, v)
     kk = min(p.k, v)
     mm = min(p.m, max(0, v - p.k))
     route = np.full(p.k, -1, np.int32)
     route[:kk] = order[:kk]
-    sent = np.full(p.m + p.r, -1, np.int32)
+    sent = np.full(p.sw, -1, np.int32)
     sent[:mm] = order[kk:kk + mm]
-    rand = draw_random_sentinels(list(order[:kk + mm]), v, p.r, p.seed, g, layer)
+    excluded = [int(j) for j in order[:kk + mm]]
+    wanted = ([0] if p.global_sentinels & 1 else []) + ([v - 1] if p.global_sentinels & 2 else [])
+    for slot, j in enumerate(wanted):
+        if v > 0 and j not in excluded:
+            sent[p.m + p.r + slot] = j
+            excluded.append(j)
+    rand = draw_random_sentinels(excluded, v, p.r, p.seed, g, layer)
     sent[p.m:p.m + len(rand)] = rand
     kth = float(s_row[order[kk - 1]])
     margin = float(kth - s_row[order[kk]]) if v > kk else float("inf")
@@ -296,8 +327,17 @@ def relay_layer(prev: Ledger, q: np.ndarray, k: np.ndarray, p: OracleParams, lay
         beta[sl] = b
         reuse = np.zeros(p.n_q, bool)
         for i in range(p.n_q):
-            # Eq. 5: reuse iff alpha > beta + gamma; a row without sentinels is never flagged
-            reuse[i] = (not has_sent[i]) or bool(a[i] > b[i] + p.gamma)
+            age = int(prev.ages[sl][i])
+            # guard margin of the row: larger while the margin recorded at its last routing is
+            # below the recovery level (decided in float32, the precision the ledger stores)
+            weak = bool(np.float32(prev.margin[sl][i]) < np.float32(p.margin_recover))
+            gamma_i = p.gamma + (p.gamma_boost if weak else 0.0)
+            # Eq. 5: reuse iff alpha > beta + gamma_i; a row without sentinels is never flagged
+            reuse[i] = (not has_sent[i]) or bool(a[i] > b[i] + gamma_i)
+            if age < p.min_reuse:              # minimum reuse horizon: not tested yet
+                reuse[i] = True
+            if p.h_max > 0 and age >= p.h_max:  # forced re-routing of an old route
+                reuse[i] = False
         flags[sl] = (~reuse).astype(np.uint8)
     refresh_rows = np.nonzero(flags)[0].astype(np.int64)       # ascending = prefix-sum order
     for gr in refresh_rows:

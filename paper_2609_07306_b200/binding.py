@@ -37,7 +37,9 @@ class rr_config(C.Structure):
                 ("n_k", C.c_int32), ("d", C.c_int32), ("k", C.c_int32), ("m", C.c_int32),
                 ("r", C.c_int32), ("dtype", C.c_int32), ("causal", C.c_int32),
                 ("causal_offset", C.c_int32), ("gamma", C.c_float), ("seed", C.c_uint64),
-                ("chunk_tokens", C.c_int32), ("debug_outputs", C.c_int32)]
+                ("chunk_tokens", C.c_int32), ("debug_outputs", C.c_int32),
+                ("global_sentinels", C.c_int32), ("min_reuse", C.c_int32), ("h_max", C.c_int32),
+                ("gamma_boost", C.c_float), ("margin_recover", C.c_float)]
 
 
 class rr_views(C.Structure):

@@ -46,7 +46,11 @@ int validate(const rr_config* c) {
   if (c->d != 64 && c->d != 128) return RR_ERR_UNSUPPORTED;
   if (c->n_k > RR_MAX_NK) return RR_ERR_UNSUPPORTED;
   if (c->k > c->n_k) return RR_ERR_INVALID_ARG;
-  if (c->k + c->m + c->r > RR_MAX_C) return RR_ERR_UNSUPPORTED;
+  if (c->global_sentinels < 0 || c->global_sentinels > 3) return RR_ERR_INVALID_ARG;
+  if (c->min_reuse < 0 || c->h_max < 0 || !(c->gamma_boost >= 0.f)) return RR_ERR_INVALID_ARG;
+  if (c->margin_recover != c->margin_recover) return RR_ERR_INVALID_ARG;   // NaN
+  if (c->k + c->m + c->r + (c->global_sentinels & 1) + ((c->global_sentinels >> 1) & 1) > RR_MAX_C)
+    return RR_ERR_UNSUPPORTED;
   const long long rows = (long long)c->batch * c->heads * c->n_q;
   if (rows > (1LL << 30)) return RR_ERR_UNSUPPORTED;
   if (c->chunk_tokens > 0 && (long long)c->n_k * c->chunk_tokens > 0x7FFFFFFFLL)
@@ -58,7 +62,12 @@ int validate(const rr_config* c) {
 RRParams shape_params(const rr_config* cfg) {
   RRParams p{};
   p.P = cfg->batch * cfg->heads; p.n_q = cfg->n_q; p.n_k = cfg->n_k; p.d = cfg->d;
-  p.k = cfg->k; p.m = cfg->m; p.r = cfg->r; p.sw = cfg->m + cfg->r; p.c = cfg->k + p.sw;
+  p.k = cfg->k; p.m = cfg->m; p.r = cfg->r;
+  p.global_mask = cfg->global_sentinels;
+  p.n_global = (cfg->global_sentinels & 1) + ((cfg->global_sentinels >> 1) & 1);
+  p.min_reuse = cfg->min_reuse; p.h_max = cfg->h_max;
+  p.gamma_boost = cfg->gamma_boost; p.margin_recover = cfg->margin_recover;
+  p.sw = cfg->m + cfg->r + p.n_global; p.c = cfg->k + p.sw;
   p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
   p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs & 1;
   p.rows = p.P * p.n_q;
@@ -75,7 +84,8 @@ bool uses_fused(const rr_config* cfg) {
 Layout make_layout(const rr_config* c) {
   Layout L{};
   const size_t P = (size_t)c->batch * c->heads, rows = P * c->n_q;
-  const size_t sw = (size_t)c->m + c->r, cw = (size_t)c->k + sw;
+  const size_t sw = (size_t)c->m + c->r + (c->global_sentinels & 1) + ((c->global_sentinels >> 1) & 1),
+               cw = (size_t)c->k + sw;
   const size_t tiles = P * ((c->n_q + RR_ROW_TILE - 1) / RR_ROW_TILE);
   size_t o = 0;
   L.routes = o;    o = align_up(o + rows * c->k * 4);

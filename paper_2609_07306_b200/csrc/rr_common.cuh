@@ -12,7 +12,9 @@
 
 // Everything a kernel needs to know about one ledger; passed by value.
 struct RRParams {
-  int P, n_q, n_k, d, k, m, r, c, sw;      // sw = m + r (sentinel row width)
+  int P, n_q, n_k, d, k, m, r, c, sw;      // sw = m + r + n_global (sentinel row width), c = k + sw
+  int global_mask, n_global, min_reuse, h_max;   // optional policies (0 = off)
+  float gamma_boost, margin_recover;
   int dtype, causal, causal_offset, chunk_tokens, debug;   // debug: bit 0 = store candidate scores
   int rows, tiles_per_problem, n_tiles;    // row tiles of RR_ROW_TILE per problem / in total
   float gamma;
@@ -79,6 +81,22 @@ __host__ __device__ __forceinline__ unsigned long long rr_row_key(unsigned long 
 __host__ __device__ __forceinline__ uint32_t rr_draw_u32(unsigned long long row_key,
                                                          uint32_t layer, uint32_t t) {
   return (uint32_t)(rr_fmix64(row_key ^ (((unsigned long long)layer << 32) | t)) >> 32);
+}
+
+// Challenge test of Eq. 5 for global row g, with the optional policies of Section 3.2: a
+// larger guard margin while the margin recorded at the row's last routing is below the
+// recovery level, no test before the minimum reuse horizon, forced re-routing of a route
+// that is h_max layers old.  Reads the ledger's ages / margins only when a policy is on.
+__device__ __forceinline__ bool rr_challenge(const RRParams& p, int g, float alpha, float beta) {
+  float gamma = p.gamma;
+  if (p.gamma_boost > 0.f && p.margin[g] < p.margin_recover) gamma += p.gamma_boost;
+  bool flag = beta > __int_as_float(0xff800000) && !(alpha > beta + gamma);
+  if (p.min_reuse > 0 || p.h_max > 0) {
+    const int age = p.ages[g];
+    if (age < p.min_reuse) flag = false;
+    if (p.h_max > 0 && age >= p.h_max) flag = true;
+  }
+  return flag;
 }
 
 // ---- launchers (one per .cu file) -------------------------------------------------------

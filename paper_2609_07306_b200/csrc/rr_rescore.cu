@@ -106,8 +106,7 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
       n_valid += __shfl_xor_sync(FULL, n_valid, off);
     }
     if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
-    const bool has_sent = bmax > ninf;
-    const bool flag = has_sent && !(amin > bmax + p.gamma);
+    const bool flag = rr_challenge(p, g, amin, bmax);
     if (lane == 0) {
       p.flags[g] = flag ? 1 : 0;
       p.alpha[g] = amin;

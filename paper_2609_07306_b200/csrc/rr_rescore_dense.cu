@@ -222,8 +222,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
       bmax = fmaxf(bmax, __uint_as_float(lds(xch_base + PITCH + r * 4u)));
       nmin = fminf(nmin, __uint_as_float(lds(xch_base + 2u * PITCH + r * 4u)));
       const bool ok = alive && row >= 0;
-      const bool has_sent = bmax > ninf;
-      const bool flag = ok && has_sent && !(amin > bmax + p.gamma);
+      const bool flag = ok && rr_challenge(p, g, amin, bmax);
       if (ok) {
         p.flags[g] = flag ? 1 : 0;
         p.alpha[g] = amin;

@@ -818,9 +818,26 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         p.kth[g] = kth;
         p.margin[g] = v > kk ? kth - next : pinf;
 
+        // ---- mandatory global sentinels (sink chunk, most recent chunk): a slot each after
+        // the random ones, empty if the chunk is already in the route or a near-miss sentinel
+        int pool = v - (nr + nn);
+        if (p.n_global) {
+          int32_t* glob = sent + p.m + p.r;
+          int gi = 0;
+          for (int b = 0; b < 2; ++b) {
+            if (!((p.global_mask >> b) & 1)) continue;
+            const int j = b == 0 ? 0 : v - 1;
+            int id = -1;
+            if (v > 0) {
+              const uint32_t wa = bm(j >> 5);
+              const uint32_t w = aux_ld(wa), bit = 1u << (j & 31);
+              if (!(w & bit)) { aux_st(wa, w | bit); id = j; --pool; }
+            }
+            glob[gi++] = id;
+          }
+        }
         // ---- random sentinels --------------------------------------------------------------
         int32_t* rnd = sent + p.m;
-        const int pool = v - (nr + nn);
         int taken = 0;
         if (p.r > 0 && pool > 0) {
           if (pool > p.r) {

@@ -133,8 +133,27 @@ topk_rows_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t laye
   __syncwarp();
 
   // random sentinels: r distinct chunks from the valid ones outside route and near-miss
+  // mandatory global sentinels (sink chunk, most recent chunk): a slot each after the random
+  // ones, empty if the chunk is already in the route or a near-miss sentinel
+  int pool = v - Tkeep;
+  if (p.n_global) {
+    int gi = 0;
+    for (int b = 0; b < 2; ++b) {
+      if (!((p.global_mask >> b) & 1)) continue;
+      const int j = b == 0 ? 0 : v - 1;
+      int id = -1;
+      if (v > 0) {
+        const uint32_t word = bitmap[j >> 5], bit = 1u << (j & 31);
+        if (!(word & bit)) { id = j; --pool; }
+        __syncwarp();
+        if (id >= 0 && lane == 0) bitmap[j >> 5] = word | bit;
+        __syncwarp();
+      }
+      if (lane == 0) sent[p.m + p.r + gi] = id;
+      ++gi;
+    }
+  }
   int32_t* rnd = sent + p.m;
-  const int pool = v - Tkeep;
   int taken = 0;
   if (p.r > 0 && pool > 0) {
     if (pool > p.r) {

@@ -18,7 +18,10 @@ def config_from_workload(w: RouteWorkload, debug_outputs: bool = False,
                        causal=1 if w.causal else 0, causal_offset=0, gamma=float(w.gamma),
                        seed=int(w.seed), chunk_tokens=int(w.chunk_tokens),
                        debug_outputs=(1 if debug_outputs else 0) | (2 if two_pass else 0) |
-                       (4 if gathered else 0))
+                       (4 if gathered else 0),
+                       global_sentinels=int(w.global_sentinels), min_reuse=int(w.min_reuse),
+                       h_max=int(w.h_max), gamma_boost=float(w.gamma_boost),
+                       margin_recover=float(w.margin_recover))
 
 
 class RouteLedger:
@@ -39,7 +42,8 @@ class RouteLedger:
                                            self.scratch_buf.data_ptr() + self._so, sb)
         self.P = cfg.batch * cfg.heads
         self.rows = self.P * cfg.n_q
-        self.c = cfg.k + cfg.m + cfg.r
+        self.sw = cfg.m + cfg.r + (cfg.global_sentinels & 1) + ((cfg.global_sentinels >> 1) & 1)
+        self.c = cfg.k + self.sw
         self._views = B.rr_ledger_views(self.handle)
         self.reset()
 
@@ -110,7 +114,7 @@ class RouteLedger:
     @property
     def routes(self): return self._view("routes", "i32", (self.rows, self.cfg.k))
     @property
-    def sentinels(self): return self._view("sentinels", "i32", (self.rows, self.cfg.m + self.cfg.r))
+    def sentinels(self): return self._view("sentinels", "i32", (self.rows, self.sw))
     @property
     def ages(self): return self._view("ages", "i32", (self.rows,))
     @property

@@ -59,6 +59,12 @@ class RouteWorkload:
     redraw_every: int = 0     # 0 = never
     redraw_frac: float = 0.0
     chunk_tokens: int = 0     # >0: routes are also expanded to token ranges
+    # optional policies (Section 3.1 item 3, Section 3.2 "Hysteresis" / "Forced anchors")
+    global_sentinels: int = 0   # bit 0: sink chunk, bit 1: most recent chunk
+    min_reuse: int = 0
+    gamma_boost: float = 0.0
+    margin_recover: float = 0.0
+    h_max: int = 0
 
     @property
     def problems(self) -> int:
@@ -69,8 +75,12 @@ class RouteWorkload:
         return self.problems * self.n_q
 
     @property
+    def sw(self) -> int:
+        return self.m + self.r + (self.global_sentinels & 1) + ((self.global_sentinels >> 1) & 1)
+
+    @property
     def c(self) -> int:
-        return self.k + self.m + self.r
+        return self.k + self.sw
 
     def is_anchor(self, layer: int) -> bool:
         return layer % self.anchor_every == 0

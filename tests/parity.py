@@ -31,7 +31,10 @@ from paper_2609_07306_b200.ledger import RouteLedger, config_from_workload, devi
 
 def oracle_params(w: W.RouteWorkload) -> O.OracleParams:
     return O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, gamma=w.gamma,
-                          causal=w.causal, causal_offset=0, seed=w.seed)
+                          causal=w.causal, causal_offset=0, seed=w.seed,
+                          global_sentinels=w.global_sentinels, min_reuse=w.min_reuse,
+                          gamma_boost=w.gamma_boost, margin_recover=w.margin_recover,
+                          h_max=w.h_max)
 
 
 def score_tol(qn: np.ndarray, kn_max: float, s_abs: np.ndarray) -> np.ndarray:
@@ -101,6 +104,7 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
             led.routes[sel_t] = torch.from_numpy(oracle_led.routes).cuda()
             led.sentinels[sel_t] = torch.from_numpy(oracle_led.sentinels).cuda()
             led.ages[sel_t] = torch.from_numpy(oracle_led.ages).cuda()
+            led.margin[sel_t] = torch.from_numpy(oracle_led.margin.astype(np.float32)).cuda()
             prev_gpu_routes = led.routes.clone()
             prev_gpu_sent = led.sentinels.clone()
             prev_gpu_ages = led.ages.clone()
@@ -170,8 +174,12 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
                 if not np.array_equal(np.isfinite(gv), fin) or \
                         (np.abs(gv[fin] - ov[fin]) > tol_row[fin]).any():
                     rep.bad(f"layer {l}: {name} differs beyond tolerance")
-            slack = np.abs(res.alpha - res.beta - p.gamma)
-            amb_flag = np.isfinite(slack) & (slack <= amb_tol)
+            weak = oracle_led.margin.astype(np.float32) < np.float32(p.margin_recover)
+            slack = np.abs(res.alpha - res.beta - (p.gamma + np.where(weak, p.gamma_boost, 0.0)))
+            tested = oracle_led.ages >= p.min_reuse          # policy rows decide without Eq. 5
+            if p.h_max > 0:
+                tested &= oracle_led.ages < p.h_max
+            amb_flag = np.isfinite(slack) & (slack <= amb_tol) & tested
             rep.ambiguous_flag_rows += int(amb_flag.sum())
             diff = g_flags != res.flags
             rep.flag_mismatch_ambiguous += int((diff & amb_flag).sum())

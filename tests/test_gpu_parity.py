@@ -267,3 +267,47 @@ def test_fixed_stride_never_flags_and_low_drift_flags_few():
     _, flg_hi, _ = run(w_hi)
     print(f"flagged fraction: low drift {flg:.3f}, high drift {flg_hi:.3f}")
     assert flg < 0.5 * flg_hi
+
+
+_POLICIES = {
+    "global_sentinels": dict(global_sentinels=3),
+    "sink_only": dict(global_sentinels=1, m=0),
+    "min_reuse": dict(min_reuse=1),
+    "gamma_boost": dict(gamma_boost=0.05, margin_recover=0.02),
+    "h_max": dict(h_max=2),
+    "all": dict(global_sentinels=3, min_reuse=1, gamma_boost=0.05, margin_recover=0.02, h_max=3),
+}
+
+
+@pytest.mark.parametrize("policy", sorted(_POLICIES))
+def test_policies_either_side_of_the_trigger(policy):
+    """Mandatory global sentinels (Section 3.1 item 3), hysteresis and per-row forced
+    re-routing (Section 3.2) against the oracle, on every kernel variant."""
+    base = W.moderate().replace(heads=3, layers=7, anchor_every=100, rho=0.2)
+    w = base.replace(**_POLICIES[policy])
+    for two_pass, gathered in ((False, False), (False, True), (True, True)):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
+        _report(rep)
+        parity.assert_clean(rep)
+    # non-causal, ragged shape, d = 64
+    w2 = W.RouteWorkload("ragged_policy", 1, 2, 200, 333, 64, 12, 8, 6, layers=5, anchor_every=100,
+                         dtype=W.DTYPE_BF16, centroids=16, rho=0.1, causal=False, seed=5,
+                         **{k_: v_ for k_, v_ in _POLICIES[policy].items() if k_ != "m"})
+    rep = parity.run_teacher_forced(w2)
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_forced_rerouting_bounds_every_age():
+    """Free-running with h_max = 3 and a single anchor: no age ever exceeds 3."""
+    w = W.moderate().replace(heads=2, layers=9, anchor_every=100, rho=0.01, h_max=3)
+    q, k = W.generate(w)
+    led = RouteLedger(config_from_workload(w))
+    worst = 0
+    for l in range(w.layers):
+        fn = led.route_anchor if w.is_anchor(l) else led.route_relay
+        fn(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        worst = max(worst, int(led.ages.max().item()))
+    led.close()
+    assert worst == 3

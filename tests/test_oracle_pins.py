@@ -350,3 +350,98 @@ def test_relay_requires_anchor():
     p = O.OracleParams(n_q=4, n_k=4, k=1, m=1, r=0)
     with pytest.raises(ValueError):
         O.relay_layer(O.Ledger.empty(4, p), np.ones((1, 4, 2)), np.ones((1, 4, 2)), p, 1)
+
+
+# ---------------------------------------------------------------- optional policies
+def test_global_sentinels_hand_case():
+    """Sink (chunk 0) and most recent chunk (v - 1) are sentinels unless already in the route
+    or among the near-miss ones; the random draw avoids them (Section 3.1, item 3)."""
+    # one row, 8 chunks, scores descending in the order 3,4,0,7,1,2,5,6
+    s = np.full(8, -np.inf)
+    for rank, j in enumerate([3, 4, 0, 7, 1, 2, 5, 6]):
+        s[j] = 10.0 - rank
+    p = O.OracleParams(n_q=1, n_k=8, k=2, m=1, r=2, global_sentinels=3)
+    route, sent, kth, margin = O.route_row(s, 8, p, g=0, layer=0)
+    assert set(route) == {3, 4}
+    assert sent[0] == 0                       # near-miss: rank 3 is chunk 0 ...
+    assert sent[3] == -1 and sent[4] == 7     # ... so the sink slot stays empty; recent = 7
+    rnd = [int(x) for x in sent[1:3]]
+    assert len(set(rnd)) == 2 and not (set(rnd) & {3, 4, 0, 7}) and all(0 <= x < 8 for x in rnd)
+    # sink not in route or near-miss: it takes its slot
+    p2 = O.OracleParams(n_q=1, n_k=8, k=2, m=0, r=0, global_sentinels=3)
+    _, sent2, _, _ = O.route_row(s, 8, p2, g=0, layer=0)
+    assert list(sent2) == [0, 7]
+    # a row that sees one chunk: it is the route, nothing is left
+    _, sent3, _, _ = O.route_row(s, 1, p2, g=0, layer=0)
+    assert list(sent3) == [-1, -1]
+    # sink and recent coincide (v = 1 is covered above; v = 3 with route {0,...}): no duplicate
+    p4 = O.OracleParams(n_q=1, n_k=8, k=1, m=0, r=0, global_sentinels=3)
+    s4 = np.array([1.0, 5.0, -np.inf, -np.inf, -np.inf, -np.inf, -np.inf, -np.inf])
+    _, sent4, _, _ = O.route_row(s4, 2, p4, g=0, layer=0)
+    assert list(sent4) == [0, -1]             # route {1}; sink 0; recent = 1 is in the route
+
+
+def _one_row_ledger(p, route, sent, age, margin):
+    led = O.Ledger.empty(1, p)
+    led.routes[0, :len(route)] = route
+    led.sentinels[0, :len(sent)] = sent
+    led.ages[0] = age
+    led.margin[0] = margin
+    return led
+
+
+def test_hysteresis_and_forced_rerouting_hand_case():
+    """d = 1, q = 1: scores are the key values.  alpha - beta = 0.5."""
+    q = np.ones((1, 1, 1)); k = np.array([[[3.0], [2.5], [1.0]]])
+    base = dict(n_q=1, n_k=3, k=1, m=1, r=0)
+    # plain Eq. 5 with gamma = 0: reuse
+    p = O.OracleParams(**base)
+    led = _one_row_ledger(p, [0], [1], age=2, margin=0.1)
+    assert O.relay_layer(led, q, k, p, 1).flags[0] == 0
+    # larger guard margin while the recorded margin is below the recovery level
+    p = O.OracleParams(**base, gamma_boost=1.0, margin_recover=0.2)
+    assert O.relay_layer(led, q, k, p, 1).flags[0] == 1
+    led_ok = _one_row_ledger(p, [0], [1], age=2, margin=0.3)
+    assert O.relay_layer(led_ok, q, k, p, 1).flags[0] == 0
+    # minimum reuse horizon: a row routed at the previous layer (age 0) is not tested
+    p = O.OracleParams(**base, gamma=1.0, min_reuse=1)
+    fresh = _one_row_ledger(p, [0], [1], age=0, margin=0.1)
+    res = O.relay_layer(fresh, q, k, p, 1)
+    assert res.flags[0] == 0 and res.ledger.ages[0] == 1
+    assert O.relay_layer(res.ledger, q, k, p, 2).flags[0] == 1      # tested one layer later
+    # forced re-routing: the route is h_max layers old
+    p = O.OracleParams(**base, h_max=3)
+    assert O.relay_layer(_one_row_ledger(p, [0], [1], age=2, margin=9.0), q, k, p, 1).flags[0] == 0
+    res = O.relay_layer(_one_row_ledger(p, [0], [1], age=3, margin=9.0), q, k, p, 1)
+    assert res.flags[0] == 1 and res.ledger.ages[0] == 0
+
+
+def test_forced_rerouting_period_closed_form():
+    """With nothing to challenge a route (m = r = 0) and h_max = 2, one anchor at layer 0:
+    every row is re-routed exactly at layers 3, 6, 9, ... and nowhere else."""
+    w = W.tiny().replace(m=0, r=0, layers=10, anchor_every=100, h_max=2)
+    q, k = W.generate(w)
+    p = O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=0, r=0, h_max=2)
+    res, _ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),
+                          p, w.anchor_every)
+    for l in range(1, w.layers):
+        assert res[l].flags.all() == (l % 3 == 0) and res[l].flags.any() == (l % 3 == 0)
+        if l % 3 == 0:
+            assert np.array_equal(res[l].ledger.routes, res[l].full_routes)
+    assert max(int(r_.ledger.ages.max()) for r_ in res) == 2
+
+
+def test_minimum_reuse_horizon_invariant():
+    """A row re-routed at layer l is never flagged at layer l + 1 when min_reuse = 1."""
+    w = W.moderate().replace(heads=2, layers=8, anchor_every=100, rho=0.3, min_reuse=1)
+    q, k = W.generate(w)
+    p = O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, causal=True, min_reuse=1)
+    res, _ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),
+                          p, w.anchor_every)
+    assert res[1].flags.sum() == 0                       # the layer after the anchor
+    seen = 0
+    for l in range(2, w.layers):
+        both = (res[l - 1].flags != 0) & (res[l].flags != 0)
+        assert not both.any()
+        seen += int(res[l].flags.sum())
+    assert seen > 0
