@@ -352,6 +352,32 @@ __device__ __forceinline__ int compact_exact(const Sel& s, int n, float s_T, int
   return (int)((waddr - s.buf) / ENTRY_PITCH);
 }
 
+// The final cut and the route / near-miss split are finished on short side lists: while the
+// last pass drops what lies below the bin of rank keep, it copies the scores of that bin, and
+// of the bin of rank kk, into two lists of up to LMAX words each (in the histogram words, which
+// are dead once the bins have been scanned).  The wanted rank inside such a list is then found
+// by counting, list order breaking ties (the lists keep the buffer's ascending chunk ids).
+constexpr int LMAX = NB / 2;
+__device__ __forceinline__ void rank_in_list(uint32_t list, int cnt, int cmax, int T, float& s_T,
+                                             int& need) {
+  const int last = max(cnt - 1, 0);
+  for (int i = 0; i < cmax; ++i) {
+    const float si = ld_score(list + min(i, last) * AUX_PITCH);
+    int gt = 0, eq = 0;
+    for (int j0 = 0; j0 < cmax; j0 += 4) {
+      float sj[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sj[j] = ld_score(list + min(j0 + j, last) * AUX_PITCH);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool in = j0 + j < cnt;
+        gt += in & (sj[j] > si); eq += in & (sj[j] == si);
+      }
+    }
+    if (i < cnt && gt < T && T <= gt + eq) { s_T = si; need = T - gt; }
+  }
+}
+
 // Per-row state of the streaming threshold filter.
 struct RowState {
   float tau;          // pass threshold of the filter (inclusive)
@@ -370,9 +396,14 @@ struct RowState {
 // rebuilt at the next call.
 // FINAL: the last call of a row.  The cut is made exact (n becomes `keep`), and the same
 // level also locates rank `kk` (the route / near-miss split): s_k and need_k are returned.
+// With `lists` (FINAL only) the exact cut is not applied to the buffer: the buffer keeps the
+// entries of bin b* and above, and (s_cut, need_cut) say which of them belong to the top keep
+// (scores > s_cut, and the first need_cut entries equal to it); lanes that had to take the
+// slow way return s_cut = -inf (everything left in the buffer belongs).
 template <bool FINAL>
 __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_limit, RowState& st,
-                          int kk, float& s_k, int& need_k) {
+                          int kk, float& s_k, int& need_k, bool lists, float& s_cut,
+                          int& need_cut) {
   // (1) map (first call) + binning of the new entries.  With d = mean - min of the buffered
   // scores the map covers [mean - 0.5 d, mean + 1.3 d]: the cut lies around or above the mean,
   // and a few far outliers (e.g. a row's own cluster) would otherwise stretch the bins;
@@ -406,7 +437,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   const bool usable = active && st.smax > st.smin && st.map_scale > 0.f && st.map_scale < 1e37f;
   const int from = usable ? st.binned : 0, to = usable ? n : 0;
   const int nw_new = warp_max(to - from);
-  const float mlo = st.map_lo, msc = st.map_scale;
+  float mlo = st.map_lo, msc = st.map_scale;
   for (int e0 = 0; e0 < nw_new; e0 += BATCH) {
     float v[BATCH];
 #pragma unroll
@@ -428,9 +459,85 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   bc.reset(); bk.reset();
   const int nd = usable ? n : 0;
   const int nw = warp_max(nd);
+  if (FINAL && lists) {
+    // The persistent map was laid out for the row's whole score distribution; by now the
+    // buffer holds its upper tail only, so the bins around the cut are crowded.  Lay a second
+    // map over the stretch from the bin of rank keep to the bin of rank kk (one bin of slack at
+    // either end catches what lies below / above) and count again: the bins of the two ranks
+    // then hold a handful of entries each.
+    const bool crowded = usable && (bc.cnt > LMAX || bk.cnt > LMAX);
+    if (__any_sync(FULL, crowded)) {
+      const float e_lo = mlo + (float)bsel / msc, e_hi = mlo + (float)(bsel_k + 1) / msc;
+      const float w = (e_hi - e_lo) * (1.0f / (float)(NB - 2));
+      const bool remap = usable && w > 0.f && (1.0f / w) < 1e37f;
+      if (remap) { mlo = e_lo - w; msc = 1.0f / w; }
+      clear_bins_if(remap, s);
+      const int nr_ = remap ? n : 0;
+      for (int e0 = 0; e0 < nw; e0 += BATCH) {
+        float v[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(nr_ - 1, 0)) * ENTRY_PITCH);
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+          const bool in = e0 + j < nr_;
+          const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+          const uint32_t a = s.aux + b * AUX_PITCH;
+          aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+        }
+      }
+      int b1, b2; BinInfo t1, t2;
+      scan_bins(s, keep, b1, t1.cnt, t1.above);
+      scan_bins(s, kk, b2, t2.cnt, t2.above);
+      if (remap) { bsel = b1; bsel_k = b2; bc.cnt = t1.cnt; bc.above = t1.above; bk.cnt = t2.cnt; bk.above = t2.above; }
+    }
+  }
   uint32_t waddr = s.buf;
   // bin >= bsel  <=>  (v - lo) * scale >= bsel for bsel >= 1; bin 0 also holds what lies below lo
   const float tb = bsel == 0 ? __int_as_float(0xff800000) : (float)bsel;
+  // FINAL, every lane with work has a usable map and short bins: side lists instead of tracking
+  const bool fast_lane = FINAL && lists && usable && bc.cnt <= LMAX && bk.cnt <= LMAX;
+  const bool fast = FINAL && lists && __all_sync(FULL, fast_lane || !active);
+#ifdef RR_PHASE_TIMING
+  if (FINAL) {
+    const int n_slow_lanes = __popc(__ballot_sync(FULL, active && !fast_lane));
+    const int worst = warp_max(active ? max(bc.cnt, bk.cnt) : 0);
+    PH_CNT(13, fast ? 1 : 0); PH_CNT(14, n_slow_lanes); PH_CNT(15, worst);
+  }
+#endif
+  if (fast) {
+    const uint32_t list_c = s.aux, list_k = s.aux + LMAX * AUX_PITCH;
+    uint32_t wc = list_c, wk = list_k;
+    for (int e0 = 0; e0 < nw; e0 += BATCH) {
+      float v[BATCH]; uint32_t id[BATCH];
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j)
+        ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) {
+        const float t = (v[j] - mlo) * msc;
+        const bool live = e0 + j < nd;
+        const bool keep_it = live & (t >= tb);
+        const int b = max(0, min(NB - 1, __float2int_rz(t)));
+        const bool in_c = live & (b == bsel), in_k = live & (b == bsel_k);
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                     ::"r"(wc), "f"(v[j]), "r"((uint32_t)in_c) : "memory");
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                     ::"r"(wk), "f"(v[j]), "r"((uint32_t)in_k) : "memory");
+        wc += in_c ? AUX_PITCH : 0u; wk += in_k ? AUX_PITCH : 0u;
+        st_entry_if(keep_it, waddr, v[j], id[j]);
+        waddr += keep_it ? ENTRY_PITCH : 0u;
+      }
+    }
+    if (active) n = (int)((waddr - s.buf) / ENTRY_PITCH);
+    const int cnt_c = active ? bc.cnt : 0, cnt_k = active ? bk.cnt : 0;
+    s_cut = __int_as_float(0xff800000); need_cut = 0;
+    rank_in_list(list_c, cnt_c, warp_max(cnt_c), keep - bc.above, s_cut, need_cut);
+    float ks = 0.f; int kn = 0;
+    rank_in_list(list_k, cnt_k, warp_max(cnt_k), kk - bk.above, ks, kn);
+    if (active) { s_k = ks; need_k = kn; }
+    return;
+  }
+  if (FINAL) { s_cut = __int_as_float(0xff800000); need_cut = 0; }
   for (int e0 = 0; e0 < nw; e0 += BATCH) {
     float v[BATCH]; uint32_t id[BATCH];
 #pragma unroll
@@ -467,7 +574,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     const int nz = __popc(__ballot_sync(FULL, zoom)), nu = __popc(__ballot_sync(FULL, active && !usable));
     const int ndr = __popc(__ballot_sync(FULL, zoom && bsel == 0));
     const int ntop = __popc(__ballot_sync(FULL, zoom && bsel == NB - 1));
-    PH_CNT(13, nz); PH_CNT(14, ntop); PH_CNT(15, ndr);
+    (void)nz; (void)ntop; (void)ndr;
   }
 #endif
   if (__any_sync(FULL, zoom)) {
@@ -686,7 +793,8 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
             int n = (int)((waddr - sel.buf) / ENTRY_PITCH);
             const bool act = n > keep;
             float dummy_s; int dummy_n;
-            retighten<false>(sel, act, n, keep, (keep + cap - CHUNK) / 2, st, 0, dummy_s, dummy_n);
+            retighten<false>(sel, act, n, keep, (keep + cap - CHUNK) / 2, st, 0, dummy_s, dummy_n,
+                             false, dummy_s, dummy_n);
             if (act) waddr = sel.buf + (uint32_t)n * ENTRY_PITCH;
             PH_ADD(1); PH_CNT(8, 1);
           }
@@ -728,6 +836,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       PH_CNT(11, 1);
       // ---- exact cut at rank keep and split at rank kk (entries <= keep: nothing to cut) ----------
       float s_k = ninf; int need_k = 0;        // defaults: everything buffered is selected
+      float s_cut = ninf; int need_cut = 0;    // ... and everything buffered belongs to the top keep
       {
         PH_T0();
         if (__any_sync(FULL, n > kk)) {
@@ -736,7 +845,10 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
             // over the whole buffer (no map was ever needed for them)
           }
           const bool cut = n > keep;
-          retighten<true>(sel, cut, n, keep, -1, st, kk, s_k, need_k);
+          // the side lists live in the histogram words, which also hold the exclusion bitmap
+          // unless that sits in the buffer tail (where entries beyond keep would be in its way)
+          retighten<true>(sel, cut, n, keep, -1, st, kk, s_k, need_k, aux_words <= NB, s_cut,
+                          need_cut);
           // rows with kk < n <= keep never enter the cut: split them over the whole buffer
           const bool small = !cut && n > kk;
           if (__any_sync(FULL, small)) {
@@ -765,7 +877,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       // of slots 0.., near-miss ids in the id word of slots 0.. (a slot is only overwritten
       // after its entry has been read); the exclusion bitmap is written word by word, which
       // works because the entries are in ascending chunk id.
-      int nr = 0, nn = 0, ties = 0, cur_word = 0;
+      int nr = 0, nn = 0, ties = 0, ties_cut = 0, cur_word = 0;
       uint32_t cur_bits = 0u;
       float kth = pinf, next = ninf;
       const int nw = warp_max(n);
@@ -776,7 +888,9 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           ld_entry(sel.buf + min(e0 + j, max(n - 1, 0)) * ENTRY_PITCH, sv[j], id[j]);
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
-          const bool live = e0 + j < n;
+          const bool eq_cut = (e0 + j < n) & (sv[j] == s_cut);
+          const bool live = (e0 + j < n) & ((sv[j] > s_cut) | (eq_cut & (ties_cut < need_cut)));
+          ties_cut += eq_cut;
           const bool eq = live & (sv[j] == s_k);
           const bool in_route = live & ((sv[j] > s_k) | (eq & (ties < need_k)));
           const bool in_near = live & !in_route & (nn < p.m);
