@@ -378,11 +378,29 @@ __device__ __forceinline__ void rank_in_list(uint32_t list, int cnt, int cmax, i
   }
 }
 
+// Smallest and largest score in the lane's buffer (lanes with n = 0 get +inf / -inf).
+__device__ __forceinline__ void buffer_minmax(const Sel& s, int n, float& mn, float& mx) {
+  const int nw = warp_max(n);
+  mn = __int_as_float(0x7f800000); mx = __int_as_float(0xff800000);
+  for (int e0 = 0; e0 < nw; e0 += BATCH) {
+    float v[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(n - 1, 0)) * ENTRY_PITCH);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      mn = fminf(mn, n > 0 ? v[j] : mn); mx = fmaxf(mx, n > 0 ? v[j] : mx);
+    }
+  }
+}
+// Upper end of a search range when only a lower bound of the buffered scores is known: the
+// first level then puts everything into one bin and the next one zooms into the real range.
+constexpr float kNoUpperBound = 3.0e38f;
+
 // Per-row state of the streaming threshold filter.
 struct RowState {
   float tau;          // pass threshold of the filter (inclusive)
   float blo;          // lower bound of the buffered scores
-  float smin, smax;   // smallest buffered score so far / largest valid score seen
+  float smin, smax;   // smallest / largest buffered score when the map was laid out
   float map_lo, map_scale;   // fixed score -> bin map of the persistent histogram
   int binned;         // buffer entries [0, binned) are counted in the histogram; -1: no map yet
 };
@@ -412,15 +430,19 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   if (__any_sync(FULL, fresh)) {
     const int nf = fresh ? n : 0;
     const int nwf = warp_max(nf);
-    float sum = 0.f;
+    float sum = 0.f, mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);
     for (int e0 = 0; e0 < nwf; e0 += BATCH) {
       float v[BATCH];
 #pragma unroll
       for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(nf - 1, 0)) * ENTRY_PITCH);
 #pragma unroll
-      for (int j = 0; j < BATCH; ++j) sum += e0 + j < nf ? v[j] : 0.f;
+      for (int j = 0; j < BATCH; ++j) {      // indices past nf re-read the last entry: harmless
+        sum += e0 + j < nf ? v[j] : 0.f;
+        mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]);
+      }
     }
     if (fresh) {
+      st.smin = mn; st.smax = mx;
       const float mean = sum / (float)max(nf, 1);
       const float d = mean - st.smin;
       // full distribution buffered (no threshold yet): skip its lower tail; a buffer that was
@@ -435,6 +457,10 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     }
   }
   const bool usable = active && st.smax > st.smin && st.map_scale > 0.f && st.map_scale < 1e37f;
+  // lanes without a usable map (all buffered scores equal, or a range too narrow to scale)
+  // search their whole buffer below: its exact bounds
+  float fb_lo = 0.f, fb_hi = 0.f;
+  if (__any_sync(FULL, active && !usable)) buffer_minmax(s, active && !usable ? n : 0, fb_lo, fb_hi);
   const int from = usable ? st.binned : 0, to = usable ? n : 0;
   const int nw_new = warp_max(to - from);
   float mlo = st.map_lo, msc = st.map_scale;
@@ -584,8 +610,8 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     // entries outrank it; otherwise the whole (already reduced) buffer is searched
     const bool inbin = FINAL && usable;
     select_rank(s, zoom, n, inbin ? keep - bc.above : keep, true, fit_limit,
-                inbin ? bc.mn1 : (usable ? bc.mn1 : fminf(st.blo, st.smin)),
-                inbin ? bc.mx1 : st.smax, zs, zn, zexact);
+                inbin ? bc.mn1 : (usable ? bc.mn1 : fb_lo),
+                inbin ? bc.mx1 : (usable ? kNoUpperBound : fb_hi), zs, zn, zexact);
     if (zoom) {
       if (zexact) { s_T = zs; need = zn; }
       else { st.tau = zs; st.blo = zs; }        // fits now; zs = smallest surviving score
@@ -618,7 +644,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
     if (__any_sync(FULL, kzoom)) {
       float zs; int zn; bool zexact; int n_ = n;
       select_rank(s, kzoom, n_, usable ? kk - bk.above : kk, false, -1,
-                  usable ? bk.mn1 : fminf(st.blo, st.smin), usable ? bk.mx1 : st.smax, zs, zn,
+                  usable ? bk.mn1 : fb_lo, usable ? bk.mx1 : fb_hi, zs, zn,
                   zexact);
       if (kzoom) { ks = zs; kn = zn; }
     }
@@ -806,7 +832,6 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
             for (int q = 0; q < CHUNK; ++q) {
               const float sc = __uint_as_float(acc[c][q]);
               const bool pass = sc >= tau_f;
-              st.smin = fminf(st.smin, pass ? sc : st.smin); st.smax = fmaxf(st.smax, sc);
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
               waddr += pass ? ENTRY_PITCH : 0u;
             }
@@ -816,8 +841,6 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
               const float sc = __uint_as_float(acc[c][q]);
               const bool valid = col0 + q < v;
               const bool pass = valid && sc >= tau_f;
-              st.smin = fminf(st.smin, pass ? sc : st.smin);
-              st.smax = fmaxf(st.smax, valid ? sc : st.smax);
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
               waddr += pass ? ENTRY_PITCH : 0u;
             }
@@ -853,7 +876,9 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           const bool small = !cut && n > kk;
           if (__any_sync(FULL, small)) {
             float zs; int zn; bool zexact; int n_ = n;
-            select_rank(sel, small, n_, kk, false, -1, st.smin, st.smax, zs, zn, zexact);
+            float lo_s, hi_s;
+            buffer_minmax(sel, small ? n : 0, lo_s, hi_s);
+            select_rank(sel, small, n_, kk, false, -1, lo_s, hi_s, zs, zn, zexact);
             if (small) { s_k = zs; need_k = zn; }
           }
         }
