@@ -62,12 +62,15 @@ __device__ __forceinline__ void max_if(float& acc, float s, uint32_t word, uint3
 }
 
 #ifdef RR_PHASE_TIMING
+// cycles per phase, kept in registers and added to the global totals once per warp
 __device__ unsigned long long g_rd_phase[8];
-#define RD_T0() long long rd_t0_ = clock64()
-#define RD_LAP(i) do { const long long t1_ = clock64(); if ((threadIdx.x & 31) == 0) atomicAdd(&g_rd_phase[i], (unsigned long long)(t1_ - rd_t0_)); rd_t0_ = t1_; } while (0)
+#define RD_T0() long long rd_t0_ = clock64(); long long rd_acc_[5] = {0, 0, 0, 0, 0}
+#define RD_LAP(i) do { const long long t1_ = clock64(); rd_acc_[i] += t1_ - rd_t0_; rd_t0_ = t1_; } while (0)
+#define RD_FLUSH() do { if ((threadIdx.x & 31) == 0) { for (int i_ = 0; i_ < 5; ++i_) atomicAdd(&g_rd_phase[i_], (unsigned long long)rd_acc_[i_]); } } while (0)
 #else
 #define RD_T0() do {} while (0)
 #define RD_LAP(i) do {} while (0)
+#define RD_FLUSH() do {} while (0)
 #endif
 
 // Per-row bitmaps: row r owns `pitch` = 2*words + 1 consecutive words (odd, so that the 32 rows
@@ -97,6 +100,26 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
   const int tile_id = prob * tiles_m + tm;
   if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; }
   RD_T0();
+
+  // Consumer warps fetch the ledger ids of the rows whose bitmaps they will build before
+  // anything else, so that the memory round trip overlaps the pipeline set-up.  Lane L takes
+  // candidate slots L, L+32, ... of each row: coalesced loads, all rows in flight at once.
+  const int cquarter = warp & 3, cpart = (warp - 2) >> 2;
+  const int rb = cquarter * 32 + cpart * ROWS_PER_WARP;          // first row of this warp's share
+  const int row_b = tm * tcpipe::BM + rb;
+  auto load_ids = [&](int s0, int (&ids)[ROWS_PER_WARP]) {
+    const int s = s0 + lane;
+    const bool is_route = s < p.k;
+    const int32_t* src = is_route ? p.routes + ((size_t)prob * p.n_q + row_b) * p.k + s
+                                  : p.sentinels + ((size_t)prob * p.n_q + row_b) * p.sw + (s - p.k);
+    const int stride = is_route ? p.k : p.sw;
+#pragma unroll
+    for (int j = 0; j < ROWS_PER_WARP; ++j)
+      ids[j] = (row_b + j < p.n_q && s < p.c) ? __ldg(src + (size_t)j * stride) : -1;
+  };
+  int ids0[ROWS_PER_WARP], ids1[ROWS_PER_WARP];
+  if (warp >= 2) { load_ids(0, ids0); load_ids(32, ids1); }
+
   pipe.setup(p, nullptr, &tmap_k, nullptr, prob, tm, 0, p.n_q, NT, &tmap_q);
   const int n_tiles = pipe.num_tiles(p);
 
@@ -107,7 +130,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
   } else {
     // a warp may only read the TMEM lanes 32*(warp % 4) ...: warps 2-5 take the first COLS
     // columns of their quarter's rows, warps 6-9 the rest
-    const int quarter = warp & 3, part = (warp - 2) >> 2;
+    const int quarter = cquarter, part = cpart;
     const int r = quarter * 32 + lane;
     const int row = tm * tcpipe::BM + r < p.n_q ? tm * tcpipe::BM + r : -1;   // rows are consecutive
     const int g = prob * p.n_q + tm * tcpipe::BM + r;
@@ -119,26 +142,16 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
     RD_LAP(0);
     // ---- ledger rows -> bitmaps: each warp builds ROWS_PER_WARP rows, all lanes together ------
     {
-      const int rb = quarter * 32 + part * ROWS_PER_WARP;          // first row of this warp's share
       const uint32_t wbase = bm_base + (uint32_t)rb * pitch * 4u;  // 16-byte aligned stretch
       for (uint32_t o = lane * 16u; o < (uint32_t)ROWS_PER_WARP * pitch * 4u; o += 512u)
         sts_zero16(wbase + o);
       __syncwarp();
       RD_LAP(4);
       int n_ok = 0; bool bad = false;
-      const int row_b = tm * tcpipe::BM + rb;
-      // lane L takes candidate slots L, L+32, ...: the ids of a row are read with coalesced
-      // loads, all rows in flight at once, and set with fire-and-forget shared-memory ORs
-      for (int s0 = 0; s0 < p.c; s0 += 32) {
+      // bits are set with fire-and-forget shared-memory ORs
+      auto set_bits = [&](int s0, const int (&ids)[ROWS_PER_WARP]) {
         const int s = s0 + lane;
         const bool is_route = s < p.k, is_near = !is_route && s < p.k + p.m;
-        const int32_t* src = is_route ? p.routes + ((size_t)prob * p.n_q + row_b) * p.k + s
-                                      : p.sentinels + ((size_t)prob * p.n_q + row_b) * p.sw + (s - p.k);
-        const int stride = is_route ? p.k : p.sw;
-        int ids[ROWS_PER_WARP];
-#pragma unroll
-        for (int j = 0; j < ROWS_PER_WARP; ++j)
-          ids[j] = (row_b + j < p.n_q && s < p.c) ? __ldg(src + (size_t)j * stride) : -1;
         const uint32_t plane_a = is_near ? 0u : 1u, plane_b = is_route ? 0u : 1u;
 #pragma unroll
         for (int j = 0; j < ROWS_PER_WARP; ++j) {
@@ -155,6 +168,12 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
           if (p.debug && row_b + j < p.n_q && s < p.c)
             p.cand_scores[((size_t)prob * p.n_q + row_b + j) * p.c + s] = __int_as_float(0x7fc00000);
         }
+      };
+      set_bits(0, ids0);
+      if (p.c > 32) set_bits(32, ids1);
+      for (int s0 = 64; s0 < p.c; s0 += 32) {
+        load_ids(s0, ids0);
+        set_bits(s0, ids0);
       }
       if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
       n_ok = __reduce_add_sync(FULL, n_ok);
@@ -210,6 +229,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
       RD_LAP(3);
     }
 
+    RD_FLUSH();
     // ---- the second thread of each row hands its partial results to the first ---------------
     if (part != 0) {
       sts(xch_base + r * 4u, __float_as_uint(amin));
