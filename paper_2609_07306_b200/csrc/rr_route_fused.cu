@@ -652,7 +652,10 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   }
 }
 
-template <int D>
+// STEP: scores filtered between two checks of the buffer fill.  32 (one TMEM load) unless the
+// buffer has little room above `keep` (wide routes): there a finer step lets the buffer fill
+// closer to its capacity before each re-tightening, which is worth the extra checks.
+template <int D, int STEP>
 __global__ void __launch_bounds__(NT, 1)
 route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
@@ -791,7 +794,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     st.blo = pinf; st.smin = pinf; st.smax = ninf;
     st.map_lo = 0.f; st.map_scale = 0.f; st.binned = -1;
     uint32_t waddr = sel.buf;                 // next free entry
-    const uint32_t trigger = sel.buf + (uint32_t)(cap - CHUNK) * ENTRY_PITCH;
+    const uint32_t trigger = sel.buf + (uint32_t)(cap - STEP) * ENTRY_PITCH;
     int vmaxw = v, vminw = row >= 0 ? v : 0x7FFFFFFF;
 #pragma unroll
     for (int off = 16; off; off >>= 1) {
@@ -810,8 +813,8 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         uint32_t acc[2][32];
         tmem_ld_32x64(tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN, acc[0], acc[1]);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          const int col0 = t * BN + c * CHUNK;
+        for (int c = 0; c < BN / STEP; ++c) {
+          const int col0 = t * BN + c * STEP;
           if (col0 >= vmaxw) break;
           if (__any_sync(FULL, waddr > trigger)) {
             // re-tighten: raise the threshold until the buffer fits again
@@ -819,26 +822,27 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
             int n = (int)((waddr - sel.buf) / ENTRY_PITCH);
             const bool act = n > keep;
             float dummy_s; int dummy_n;
-            retighten<false>(sel, act, n, keep, (keep + cap - CHUNK) / 2, st, 0, dummy_s, dummy_n,
+            retighten<false>(sel, act, n, keep, (keep + cap - STEP) / 2, st, 0, dummy_s, dummy_n,
                              false, dummy_s, dummy_n);
             if (act) waddr = sel.buf + (uint32_t)n * ENTRY_PITCH;
             PH_ADD(1); PH_CNT(8, 1);
           }
           PH_T0();
           const float tau_f = st.tau;
+          const uint32_t* a = &acc[c / (CHUNK / STEP)][(c % (CHUNK / STEP)) * STEP];
           // threshold filter: branch-free appends (predicated stores); waddr is the only chain
-          if (col0 + CHUNK <= vminw) {
+          if (col0 + STEP <= vminw) {
 #pragma unroll
-            for (int q = 0; q < CHUNK; ++q) {
-              const float sc = __uint_as_float(acc[c][q]);
+            for (int q = 0; q < STEP; ++q) {
+              const float sc = __uint_as_float(a[q]);
               const bool pass = sc >= tau_f;
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
               waddr += pass ? ENTRY_PITCH : 0u;
             }
           } else {
 #pragma unroll
-            for (int q = 0; q < CHUNK; ++q) {
-              const float sc = __uint_as_float(acc[c][q]);
+            for (int q = 0; q < STEP; ++q) {
+              const float sc = __uint_as_float(a[q]);
               const bool valid = col0 + q < v;
               const bool pass = valid && sc >= tau_f;
               st_entry_if(pass, waddr, sc, (uint32_t)(col0 + q));
@@ -1070,22 +1074,27 @@ cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void*
   cudaError_t e = rr_encode_tmap_bf16_3d(&tmap, kc, p.d, p.n_k, p.P, BN);
   if (e != cudaSuccess) return e;
   const int grid = p.P * p.tiles_per_problem;
+  const int keep = p.k + (p.m > 0 ? p.m : 1);
+  const bool fine = cap - keep < 64;             // little room above keep: check the fill more often
   static bool attr_set = false;
   if (!attr_set) {
-    e = cudaFuncSetAttribute(route_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(route_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024);
-    if (e != cudaSuccess) return e;
+    const void* fns[4] = {(const void*)route_fused_kernel<128, 32>, (const void*)route_fused_kernel<128, 8>,
+                          (const void*)route_fused_kernel<64, 32>, (const void*)route_fused_kernel<64, 8>};
+    for (const void* fn : fns) {
+      e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+    }
     attr_set = true;
   }
-  if (p.d == 128)
-    route_fused_kernel<128><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, row_list,
-                                                    (uint32_t)layer, cap, aux);
+  const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
+  if (p.d == 128 && !fine)
+    route_fused_kernel<128, 32><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, cap, aux);
+  else if (p.d == 128)
+    route_fused_kernel<128, 8><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, cap, aux);
+  else if (!fine)
+    route_fused_kernel<64, 32><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, cap, aux);
   else
-    route_fused_kernel<64><<<grid, NT, smem, st>>>(p, (const __nv_bfloat16*)qc, tmap, row_list,
-                                                   (uint32_t)layer, cap, aux);
+    route_fused_kernel<64, 8><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, cap, aux);
   rr_count_launch();
   return cudaPeekAtLastError();
 }
