@@ -99,6 +99,21 @@ expand_kernel(RRParams p, int is_anchor) {
   if (!(is_anchor || p.flags[g] != 0)) return;       // stable row: ranges unchanged
   const int32_t* route = p.routes + (size_t)g * p.k;
   int32_t* out = p.token_ranges + (size_t)g * p.k * 2;
+  // rows written by the fused routing kernel are already in ascending chunk id with the empty
+  // slots last: their ranges are a plain map of the row (8-byte stores)
+  bool ordered = true;
+  for (int s = lane; s < p.k; s += 32) {
+    const int id = route[s];
+    if (s > 0 && id >= 0) { const int prev = route[s - 1]; ordered &= prev >= 0 && prev < id; }
+  }
+  if (__all_sync(FULL, ordered)) {
+    for (int s = lane; s < p.k; s += 32) {
+      const int id = route[s];
+      reinterpret_cast<int2*>(out)[s] =
+          id >= 0 ? make_int2(id * p.chunk_tokens, (id + 1) * p.chunk_tokens) : make_int2(-1, -1);
+    }
+    return;
+  }
   int n_valid = 0;
   for (int s = lane; s < p.k; s += 32) n_valid += route[s] >= 0;
 #pragma unroll

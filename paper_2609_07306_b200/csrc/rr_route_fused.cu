@@ -28,7 +28,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int BM = 128, BN = 64, B_STAGES = 2, ACC_STAGES = 4, NT = 192;
+constexpr int BM = 128, BN = 64, B_STAGES = 1, ACC_STAGES = 4, NT = 192;
 constexpr int TMEM_COLS = ACC_STAGES * BN;
 constexpr int NB = 32, NB_LOG = 5;             // histogram bins per level
 constexpr int CHUNK = 32;                      // scores handed to a thread per TMEM load
@@ -1030,7 +1030,7 @@ bool plan(const RRParams& p, int& cap, int& aux_words, size_t& smem_bytes) {
   const size_t hist = (size_t)NB * AUX_PITCH;
   if (fixed + hist >= max_smem) return false;
   const int fit = (int)((max_smem - fixed - hist) / ENTRY_PITCH);
-  cap = keep + 96;
+  cap = keep + 112;
   if (cap > fit) cap = fit;
   if (cap < keep + CHUNK) return false;
   // a bitmap wider than the histogram lives in the buffer entries beyond `keep`
