@@ -311,3 +311,23 @@ def test_forced_rerouting_bounds_every_age():
         worst = max(worst, int(led.ages.max().item()))
     led.close()
     assert worst == 3
+
+
+def test_maximum_sizes():
+    """The limits of the interface: n_k = 4096 key chunks and k + m + r = 256 candidates per row
+    (the fused kernel cannot hold such a candidate set, so this also covers the automatic
+    fall-back to the two-pass path), and n_k = 4096 with a ledger the fused kernel does hold."""
+    w = W.RouteWorkload("max_c", 1, 1, 96, 4096, 128, 128, 64, 64, layers=3, anchor_every=100,
+                        dtype=W.DTYPE_BF16, centroids=64, rho=0.2, causal=False, seed=7)
+    rep = parity.run_teacher_forced(w)
+    _report(rep)
+    parity.assert_clean(rep)
+    w = W.RouteWorkload("max_nk", 1, 2, 160, 4096, 128, 32, 16, 16, layers=3, anchor_every=100,
+                        dtype=W.DTYPE_BF16, centroids=64, rho=0.2, causal=False, seed=8)
+    for two_pass, gathered in ((False, False), (True, True)):
+        rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
+        _report(rep)
+        parity.assert_clean(rep)
+    # one key chunk more than the interface allows is refused, not truncated
+    with pytest.raises(B.RouteRelayError):
+        B.rr_workspace_bytes(config_from_workload(w.replace(n_k=4097)))
