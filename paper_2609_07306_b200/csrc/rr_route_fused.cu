@@ -957,7 +957,18 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         } else {
           for (int e = 0; e < p.k; ++e) route[e] = e < nr ? (int)aux_ld(sel.buf + e * ENTRY_PITCH) : -1;
         }
-        for (int e = 0; e < p.m; ++e) sent[e] = e < nn ? (int)aux_ld(sel.buf + e * ENTRY_PITCH + 4u) : -1;
+        if (((p.m | p.sw) & 3) == 0) {
+          for (int q = 0; q < p.m; q += 4) {
+            int4 o;
+            o.x = q + 0 < nn ? (int)aux_ld(sel.buf + (q + 0) * ENTRY_PITCH + 4u) : -1;
+            o.y = q + 1 < nn ? (int)aux_ld(sel.buf + (q + 1) * ENTRY_PITCH + 4u) : -1;
+            o.z = q + 2 < nn ? (int)aux_ld(sel.buf + (q + 2) * ENTRY_PITCH + 4u) : -1;
+            o.w = q + 3 < nn ? (int)aux_ld(sel.buf + (q + 3) * ENTRY_PITCH + 4u) : -1;
+            *reinterpret_cast<int4*>(sent + q) = o;
+          }
+        } else {
+          for (int e = 0; e < p.m; ++e) sent[e] = e < nn ? (int)aux_ld(sel.buf + e * ENTRY_PITCH + 4u) : -1;
+        }
         p.kth[g] = kth;
         p.margin[g] = v > kk ? kth - next : pinf;
 
@@ -994,12 +1005,16 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
               for (int i = 0; i < 4; ++i)
                 j4[i] = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)(t0 + i)), (uint32_t)v);
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                if (t0 + i < limit && taken < p.r) {
-                  const uint32_t wa = bm(j4[i] >> 5);
-                  const uint32_t w = aux_ld(wa), bit = 1u << (j4[i] & 31);
-                  if (!(w & bit)) { aux_st(wa, w | bit); rnd[taken++] = j4[i]; }
-                }
+              for (int i = 0; i < 4; ++i) {              // branch-free: predicated stores
+                const bool live = (t0 + i < limit) & (taken < p.r);
+                const uint32_t wa = bm(j4[i] >> 5);
+                const uint32_t w = aux_ld(wa), bit = 1u << (j4[i] & 31);
+                const bool take = live & ((w & bit) == 0u);
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.b32 [%0], %1;\n\t}"
+                             ::"r"(wa), "r"(w | bit), "r"((uint32_t)take) : "memory");
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.global.b32 [%0], %1;\n\t}"
+                             ::"l"(rnd + taken), "r"(j4[i]), "r"((uint32_t)take) : "memory");
+                taken += take;
               }
             }
           }
