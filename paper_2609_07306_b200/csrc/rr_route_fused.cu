@@ -116,6 +116,30 @@ __device__ __forceinline__ void aux_or(uint32_t addr, uint32_t bits) {
   asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(bits) : "memory");
 }
 
+// Histogram update for a batch of entries.  The bins are private to the thread, so a plain
+// load / add / store would do, but a chain of those is serialised by the shared-memory round
+// trip of each load; shared-memory reductions measured several times slower still.  Here the
+// counts of HG entries are loaded together and entries that fall into the same bin are chained
+// in registers (a later store to the same word then carries the running total).
+constexpr int HG = 4;
+__device__ __forceinline__ void hist_add(uint32_t aux, const int (&b)[8], const uint32_t (&inc)[8]) {
+#pragma unroll
+  for (int g0 = 0; g0 < 8; g0 += HG) {
+    uint32_t a[HG], c[HG];
+#pragma unroll
+    for (int i = 0; i < HG; ++i) { a[i] = aux + (uint32_t)b[g0 + i] * AUX_PITCH; c[i] = aux_ld(a[i]); }
+    uint32_t tot[HG];
+#pragma unroll
+    for (int i = 0; i < HG; ++i) {
+      uint32_t base = c[i];
+#pragma unroll
+      for (int h = 0; h < i; ++h) base = a[h] == a[i] ? tot[h] : base;   // the latest match wins
+      tot[i] = base + inc[g0 + i];
+      aux_st(a[i], tot[i]);
+    }
+  }
+}
+
 // All passes over a buffer walk it in batches of 8 with the loads issued first: a thread's
 // passes are chains of shared-memory accesses, and with one selection warp per scheduler
 // nothing else hides that latency.  Histogram increments are fire-and-forget reductions.
@@ -215,15 +239,13 @@ __device__ __forceinline__ bool lin_level(const Sel& s, int& n, int nw, float lo
     float v[BATCH];
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(ne - 1, 0)) * ENTRY_PITCH);
+    int b[BATCH]; uint32_t inc[BATCH];
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
-      // plain read-modify-write: the bins are private to this thread, and shared-memory
-      // reductions measured several times slower than a load/add/store chain here
-      const bool in = (e0 + j < ne) & (v[j] >= lo) & (v[j] <= hi);
-      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - lo) * scale)));
-      const uint32_t a = s.aux + b * AUX_PITCH;
-      aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+      inc[j] = ((e0 + j < ne) & (v[j] >= lo) & (v[j] <= hi)) ? 1u : 0u;
+      b[j] = max(0, min(NB - 1, __float2int_rz((v[j] - lo) * scale)));
     }
+    hist_add(s.aux, b, inc);
   }
   int bsel;
   scan_bins(s, rank, bsel, bi.cnt, bi.above);
@@ -469,13 +491,13 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
 #pragma unroll
     for (int j = 0; j < BATCH; ++j)
       v[j] = ld_score(s.buf + min(from + e0 + j, max(to - 1, 0)) * ENTRY_PITCH);
+    int b[BATCH]; uint32_t inc[BATCH];
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
-      const bool in = from + e0 + j < to;
-      const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
-      const uint32_t a = s.aux + b * AUX_PITCH;
-      aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+      inc[j] = from + e0 + j < to ? 1u : 0u;
+      b[j] = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
     }
+    hist_add(s.aux, b, inc);
   }
   // (2) bin of rank keep (and of rank kk), drop what lies below the former
   BinInfo bc, bk;
@@ -503,13 +525,13 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
         float v[BATCH];
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) v[j] = ld_score(s.buf + min(e0 + j, max(nr_ - 1, 0)) * ENTRY_PITCH);
+        int b[BATCH]; uint32_t inc[BATCH];
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
-          const bool in = e0 + j < nr_;
-          const int b = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
-          const uint32_t a = s.aux + b * AUX_PITCH;
-          aux_st(a, aux_ld(a) + (in ? 1u : 0u));
+          inc[j] = e0 + j < nr_ ? 1u : 0u;
+          b[j] = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
         }
+        hist_add(s.aux, b, inc);
       }
       int b1, b2; BinInfo t1, t2;
       scan_bins(s, keep, b1, t1.cnt, t1.above);
@@ -808,6 +830,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       { PH_T0(); ready = mbar_wait(&ctl->acc_full[as], aph, abort_flag); PH_ADD(0); }
       if (!__all_sync(FULL, ready)) { alive = false; break; }
       tc_fence_after();
+      static_assert(BATCH == 8, "hist_add takes batches of 8");
       static_assert(BN == 2 * CHUNK, "a tile is two TMEM loads of 32 columns");
       if (t * BN < vmaxw) {                                // else: no row of this warp sees it
         uint32_t acc[2][32];
