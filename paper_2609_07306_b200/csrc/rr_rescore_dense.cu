@@ -6,9 +6,9 @@
 // tcgen05.mma.  This variant does the latter: the same kind of tile pipeline as the fused
 // routing kernel produces S[128 rows, 32 chunks] tiles in TMEM, and the threads of a row pick
 // out the scores of the row's candidates:
-//   * at start each warp turns ledger rows into per-row bitmaps in shared memory (two planes
-//     encoding route / near-miss / random sentinel), reading the ids with coalesced loads and
-//     setting bits with shared-memory OR reductions;
+//   * at start the two threads of a row turn its ledger row into a bitmap in shared memory (two
+//     planes encoding route / near-miss / random sentinel, one plane per thread), reading the
+//     ids with 16-byte loads and setting bits with grouped read-modify-writes;
 //   * per tile a thread reads its share of the row's scores from TMEM and takes masked minima /
 //     maxima under the tile's bitmap words: alpha = min over route bits, beta = max over
 //     sentinel bits, floor = min over route and near-miss bits (the refresh's warm-start
@@ -31,7 +31,6 @@ namespace {
 constexpr int BN = 32, B_STAGES = 3, ACC_STAGES = 4;
 constexpr int TPR = 2, COLS = BN / TPR;             // threads per row, columns per thread
 constexpr int NCONS = tcpipe::BM * TPR, NT = 64 + NCONS;
-constexpr int ROWS_PER_WARP = 32 / TPR;             // ledger rows a warp turns into bitmaps
 constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr uint32_t PITCH = tcpipe::BM * 4;          // debug score column: one word per row
 
@@ -40,13 +39,6 @@ __device__ __forceinline__ uint32_t lds(uint32_t a) {
 }
 __device__ __forceinline__ void sts(uint32_t a, uint32_t v) {
   asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-// no memory clobber: the loads of the next rows' ids may move across it
-__device__ __forceinline__ void red_or(uint32_t a, uint32_t v) {
-  asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(a), "r"(v));
-}
-__device__ __forceinline__ void sts_zero16(uint32_t a) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
 }
 __device__ __forceinline__ void consumers_sync() {            // the NCONS consumer threads only
   asm volatile("bar.sync 1, %0;" ::"n"(NCONS) : "memory");
@@ -74,8 +66,7 @@ __device__ unsigned long long g_rd_phase[8];
 #endif
 
 // Per-row bitmaps: row r owns `pitch` = 2*words + 1 consecutive words (odd, so that the 32 rows
-// of a warp fall into 32 different banks when each thread reads word t of its own row, and the
-// words of one row fall into different banks when a warp builds that row together).
+// of a warp fall into 32 different banks whenever each thread touches a word of its own row).
 // Two planes encode the three candidate classes of a chunk:
 //   plane A | plane B :  route = 1|0,  near-miss = 0|1,  random sentinel = 1|1.
 template <int D>
@@ -101,24 +92,41 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
   if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; }
   RD_T0();
 
-  // Consumer warps fetch the ledger ids of the rows whose bitmaps they will build before
-  // anything else, so that the memory round trip overlaps the pipeline set-up.  Lane L takes
-  // candidate slots L, L+32, ... of each row: coalesced loads, all rows in flight at once.
+  // ---- who builds what ---------------------------------------------------------------------
+  // Each row has two consumer threads (warps 2-5: part 0, warps 6-9: part 1).  Part 0 owns
+  // plane A of its row's bitmap (route and random / global sentinels), part 1 owns plane B
+  // (all sentinels), so the two never write the same word and plain read-modify-writes do.
+  // A thread reads its ids 16 at a time (16-byte loads where the ledger row allows) and ORs
+  // them in groups of four: the four words are loaded together and ids that fall into the same
+  // word are chained in registers.  The first two batches are fetched before the pipeline
+  // set-up so that their memory round trip overlaps it.
   const int cquarter = warp & 3, cpart = (warp - 2) >> 2;
-  const int rb = cquarter * 32 + cpart * ROWS_PER_WARP;          // first row of this warp's share
-  const int row_b = tm * tcpipe::BM + rb;
-  auto load_ids = [&](int s0, int (&ids)[ROWS_PER_WARP]) {
-    const int s = s0 + lane;
-    const bool is_route = s < p.k;
-    const int32_t* src = is_route ? p.routes + ((size_t)prob * p.n_q + row_b) * p.k + s
-                                  : p.sentinels + ((size_t)prob * p.n_q + row_b) * p.sw + (s - p.k);
-    const int stride = is_route ? p.k : p.sw;
+  const int crow_l = cquarter * 32 + lane;                       // row inside the tile
+  const int crow = tm * tcpipe::BM + crow_l;
+  const bool chas = warp >= 2 && crow < p.n_q;
+  const size_t cg = (size_t)prob * p.n_q + crow;
+  // part 0: range 0 = route [0, k), range 1 = sentinel slots [m, sw); part 1: range 0 = [0, sw)
+  const int32_t* const ptr0 = cpart == 0 ? p.routes + cg * p.k : p.sentinels + cg * p.sw;
+  const int32_t* const ptr1 = p.sentinels + cg * p.sw + p.m;
+  const int n0 = chas ? (cpart == 0 ? p.k : p.sw) : 0, n1 = chas && cpart == 0 ? p.sw - p.m : 0;
+  auto load16 = [&](const int32_t* ptr, int s0, int n, int (&ids)[16]) {
+    if (s0 + 16 <= n && (((uintptr_t)(ptr + s0)) & 15u) == 0) {
 #pragma unroll
-    for (int j = 0; j < ROWS_PER_WARP; ++j)
-      ids[j] = (row_b + j < p.n_q && s < p.c) ? __ldg(src + (size_t)j * stride) : -1;
+      for (int q = 0; q < 4; ++q) {
+        const int4 t = __ldg(reinterpret_cast<const int4*>(ptr + s0) + q);
+        ids[4 * q] = t.x; ids[4 * q + 1] = t.y; ids[4 * q + 2] = t.z; ids[4 * q + 3] = t.w;
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < 16; ++q) ids[q] = s0 + q < n ? __ldg(ptr + s0 + q) : -1;
+    }
   };
-  int ids0[ROWS_PER_WARP], ids1[ROWS_PER_WARP];
-  if (warp >= 2) { load_ids(0, ids0); load_ids(32, ids1); }
+  // second prefetched batch: range 1 if the thread has one, else the next 16 of range 0
+  const bool pre1_is1 = n1 > 0;
+  const int pre1_s0 = pre1_is1 ? 0 : 16;
+  int pre0[16], pre1[16];
+  load16(ptr0, 0, n0, pre0);
+  load16(pre1_is1 ? ptr1 : ptr0, pre1_s0, pre1_is1 ? n1 : n0, pre1);
 
   pipe.setup(p, nullptr, &tmap_k, nullptr, prob, tm, 0, p.n_q, NT, &tmap_q);
   const int n_tiles = pipe.num_tiles(p);
@@ -131,50 +139,61 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
     // a warp may only read the TMEM lanes 32*(warp % 4) ...: warps 2-5 take the first COLS
     // columns of their quarter's rows, warps 6-9 the rest
     const int quarter = cquarter, part = cpart;
-    const int r = quarter * 32 + lane;
-    const int row = tm * tcpipe::BM + r < p.n_q ? tm * tcpipe::BM + r : -1;   // rows are consecutive
-    const int g = prob * p.n_q + tm * tcpipe::BM + r;
+    const int r = crow_l;
+    const int row = crow < p.n_q ? crow : -1;                       // rows are consecutive
+    const int g = (int)cg;
     const int v = row >= 0 ? rr_valid_count(row, p.n_k, p.causal, p.causal_offset) : 0;
     const uint32_t bA = bm_base + r * pitch * 4u, bB = bA + words * 4u;
     const uint32_t col = sc_base + r * 4u;
     const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
 
     RD_LAP(0);
-    // ---- ledger rows -> bitmaps: each warp builds ROWS_PER_WARP rows, all lanes together ------
+    // ---- ledger row -> this thread's plane of the row's bitmap -----------------------------
     {
-      const uint32_t wbase = bm_base + (uint32_t)rb * pitch * 4u;  // 16-byte aligned stretch
-      for (uint32_t o = lane * 16u; o < (uint32_t)ROWS_PER_WARP * pitch * 4u; o += 512u)
-        sts_zero16(wbase + o);
-      __syncwarp();
+      const uint32_t plane = part == 0 ? bA : bB;
+      for (int w = 0; w < words; ++w) sts(plane + w * 4u, 0u);
       RD_LAP(4);
       int n_ok = 0; bool bad = false;
-      // bits are set with fire-and-forget shared-memory ORs
-      auto set_bits = [&](int s0, const int (&ids)[ROWS_PER_WARP]) {
-        const int s = s0 + lane;
-        const bool is_route = s < p.k, is_near = !is_route && s < p.k + p.m;
-        const uint32_t plane_a = is_near ? 0u : 1u, plane_b = is_route ? 0u : 1u;
+      // candidates are charged once: part 0 counts what it sets, part 1 only the near-miss slots
+      auto or_ids = [&](const int (&ids)[16], int s0, int count_below) {
 #pragma unroll
-        for (int j = 0; j < ROWS_PER_WARP; ++j) {
-          const int vj = rr_valid_count(row_b + j, p.n_k, p.causal, p.causal_offset);
-          const int id = ids[j];
-          bad |= id >= vj;
-          if (id >= 0 && id < vj) {
-            const uint32_t a = wbase + ((uint32_t)j * pitch + (uint32_t)(id >> 5)) * 4u;
-            const uint32_t bit = 1u << (id & 31);
-            if (plane_a) red_or(a, bit);
-            if (plane_b) red_or(a + words * 4u, bit);
-            ++n_ok;
+        for (int g0 = 0; g0 < 16; g0 += 4) {
+          uint32_t a[4], c[4], bit[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int id = ids[g0 + i];
+            bad |= id >= v;
+            const bool ok = id >= 0 && id < v;
+            a[i] = plane + (ok ? (uint32_t)(id >> 5) * 4u : 0u);
+            bit[i] = ok ? 1u << (id & 31) : 0u;
+            n_ok += ok && s0 + g0 + i < count_below;
+            c[i] = lds(a[i]);
           }
-          if (p.debug && row_b + j < p.n_q && s < p.c)
-            p.cand_scores[((size_t)prob * p.n_q + row_b + j) * p.c + s] = __int_as_float(0x7fc00000);
+          uint32_t tot[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint32_t base = c[i];
+#pragma unroll
+            for (int h = 0; h < i; ++h) base = a[h] == a[i] ? tot[h] : base;
+            tot[i] = base | bit[i];
+            sts(a[i], tot[i]);
+          }
         }
       };
-      set_bits(0, ids0);
-      if (p.c > 32) set_bits(32, ids1);
-      for (int s0 = 64; s0 < p.c; s0 += 32) {
-        load_ids(s0, ids0);
-        set_bits(s0, ids0);
+      const int cb0 = part == 0 ? 0x7fffffff : p.m;       // range 0: all / the near-miss slots
+      or_ids(pre0, 0, cb0);
+      or_ids(pre1, pre1_s0, pre1_is1 ? 0x7fffffff : cb0);
+      const int n0_max = __reduce_max_sync(FULL, n0), n1_max = __reduce_max_sync(FULL, n1);
+      for (int s0 = pre1_is1 ? 16 : 32; s0 < n0_max; s0 += 16) {
+        load16(ptr0, s0, n0, pre0);
+        or_ids(pre0, s0, cb0);
       }
+      for (int s0 = 16; s0 < n1_max; s0 += 16) {
+        load16(ptr1, s0, n1, pre0);
+        or_ids(pre0, s0, 0x7fffffff);
+      }
+      if (p.debug && part == 0 && row >= 0)
+        for (int s = 0; s < p.c; ++s) p.cand_scores[(size_t)g * p.c + s] = __int_as_float(0x7fc00000);
       if (__any_sync(FULL, bad) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
       n_ok = __reduce_add_sync(FULL, n_ok);
       if (lane == 0) atomicAdd(&s_cnt[1], (unsigned long long)n_ok);
