@@ -43,9 +43,15 @@ def _peaks():
                 source="fallback")
 
 
+L2_BYTES = 126 << 20
+
+
 def _workload(name: str) -> W.RouteWorkload:
     if name == "sweep1024":
         return W.sweep(1024, 0.30)
+    if name.startswith("sweep_"):                     # sweep_<n>_<rho>, e.g. sweep_256_0.15
+        _, n, rho = name.split("_")
+        return W.sweep(int(n), float(rho))
     return W.PRESETS[name]()
 
 
@@ -284,17 +290,49 @@ def run_ours(args) -> None:
     # ---- timed region: device-resident inputs ----------------------------------------------
     for _ in range(args.warmup):
         step()
+    timed_step, launches_per_replay = step, None
+    if args.graph:                       # one capture of the whole step, replayed K times
+        torch.cuda.synchronize(dev)
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(dev)
+        n0 = B.rr_kernel_launch_count()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+        launches_per_replay = B.rr_kernel_launch_count() - n0    # kernels recorded in the graph
+        timed_step = graph.replay
+        for _ in range(args.warmup):
+            timed_step()
     barrier()
     clocks = ClockSampler(local)
     launches0 = B.rr_kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    # L2: a step reads every layer's inputs once.  Where one step's inputs exceed L2 several
+    # times over nothing survives from step to step; smaller workloads get L2 flushed (a
+    # 256 MB buffer written) between steps, each step timed with its own pair of events.
+    step_input_bytes = L * w.problems * (w.n_q + w.n_k) * w.d * esz
+    flush_l2 = step_input_bytes < 2 * L2_BYTES
+    if flush_l2:
+        scratch = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+        for a_ev, b_ev in evs:
+            scratch.zero_()
+            a_ev.record(stream)
+            timed_step()
+            b_ev.record(stream)
+        barrier()
+        local_ms = sum(a_ev.elapsed_time(b_ev) for a_ev, b_ev in evs)
+        del scratch
+    else:
+        e0.record(stream)
+        for _ in range(args.steps):
+            timed_step()
+        e1.record(stream)
+        barrier()
+        local_ms = e0.elapsed_time(e1)
+    ms_total = max_over_ranks(local_ms, world, dev)
     launches = B.rr_kernel_launch_count() - launches0
+    if launches_per_replay is not None:
+        launches = launches_per_replay * args.steps
     clock_info = clocks.stop()
     ms_per_step = ms_total / args.steps
     value = aggregate_rows_per_s(w.rows, L, world, ms_per_step)
@@ -428,8 +466,11 @@ def run_ours(args) -> None:
             "config": {"workload": w.name, "problems": w.problems, "n_q": w.n_q, "n_k": w.n_k,
                        "d": w.d, "k": w.k, "m": w.m, "r": w.r, "layers": L,
                        "anchor_every": w.anchor_every, "rho": w.rho, "causal": w.causal,
-                       "l2": "inputs of consecutive layers differ and exceed L2 "
-                             f"({w.problems * (w.n_q + w.n_k) * w.d * esz / 1e6:.0f} MB/layer)",
+                       "l2": ("L2 flushed between steps (256 MB written); a step's inputs are "
+                              f"{step_input_bytes / 1e6:.0f} MB" if flush_l2 else
+                              "inputs of consecutive layers differ and exceed L2 "
+                              f"({w.problems * (w.n_q + w.n_k) * w.d * esz / 1e6:.0f} MB/layer)"),
+                       "graph": bool(args.graph),
                        "host_generation_s": round(t_gen, 1)},
             "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
@@ -456,7 +497,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="high_drift",
-                    choices=sorted(W.PRESETS) + ["sweep1024"])
+                    help="one of %s, or sweep_<n>_<rho> (BASELINE configuration 3, e.g. "
+                         "sweep_256_0.15)" % ", ".join(sorted(W.PRESETS) + ["sweep1024"]))
+    ap.add_argument("--graph", action="store_true",
+                    help="time the device-resident step as replays of one CUDA graph of it "
+                         "(for the launch-bound small shapes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="truncate the layer schedule")
     ap.add_argument("--profile-only", action="store_true",

@@ -31,7 +31,7 @@ from paper_2609_07306_b200.ledger import RouteLedger, config_from_workload, devi
 
 def oracle_params(w: W.RouteWorkload) -> O.OracleParams:
     return O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, gamma=w.gamma,
-                          causal=w.causal, causal_offset=0, seed=w.seed,
+                          causal=w.causal, causal_offset=w.causal_offset, seed=w.seed,
                           global_sentinels=w.global_sentinels, min_reuse=w.min_reuse,
                           gamma_boost=w.gamma_boost, margin_recover=w.margin_recover,
                           h_max=w.h_max)

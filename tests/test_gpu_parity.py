@@ -331,3 +331,16 @@ def test_maximum_sizes():
     # one key chunk more than the interface allows is refused, not truncated
     with pytest.raises(B.RouteRelayError):
         B.rr_workspace_bytes(config_from_workload(w.replace(n_k=4097)))
+
+
+@pytest.mark.parametrize("n_q,n_k", [(384, 192), (192, 1024)])
+def test_rectangular_shapes_of_the_paper(n_q, n_k):
+    """Query and key chunk counts differ (the paper's 384 x 192 and 192 x 1024 problems),
+    without and with a causal offset that lets the last query row see every key chunk."""
+    for causal in (False, True):
+        w = W.RouteWorkload(f"rect_{n_q}x{n_k}", 1, 2, n_q, n_k, 128, 16, 8, 8, layers=4,
+                            anchor_every=100, dtype=W.DTYPE_BF16, centroids=32, rho=0.1,
+                            causal=causal, seed=11, causal_offset=max(0, n_k - n_q))
+        rep = parity.run_teacher_forced(w)
+        _report(rep)
+        parity.assert_clean(rep)
