@@ -164,7 +164,9 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
     """Algorithmic work of one kernel kind over one step, its bound and measured peak.
 
     cnt: work counters of one step (anchor_rows, relay_rows, flagged_rows, cand_pairs,
-    full_pairs).  Figures per unit are spelled out in the design doc."""
+    full_pairs).  Per unit: a routed row = 2*d*v_i FLOP of scores and (c+2)*4 bytes of ledger
+    row; a layer call reads its inputs once, P*(n_q+n_k)*d*element bytes; a relay row reads c*4
+    bytes of ledger ids and writes 13 bytes (flag, alpha, beta, tau)."""
     esz = 2 if w.dtype == W.DTYPE_BF16 else 4
     routed = cnt["anchor_rows"] + cnt["flagged_rows"]
     layer_calls = cnt["layer_calls"]

@@ -5,7 +5,8 @@
 // One CTA owns 128 query rows of one problem (consecutive rows at an anchor; a segment of the
 // compacted refresh list at a relay, Section 4.2) and walks the key chunks in tiles of 64,
 // stopping at the last chunk any of its rows may select.
-//   warp 0   : TMA producer (Kc tiles, 128-byte swizzle, 2-stage ring, no multicast)
+//   warp 0   : TMA producer (Kc tiles, 128-byte swizzle, one stage -- the selection is the slow
+//              side, so the shared memory goes to the candidate buffers --, no multicast)
 //   warp 1   : one thread issues tcgen05.mma (M=128, N=64, K=16) into a ring of 4 TMEM
 //              accumulators
 //   warps 2-5: selection, ONE THREAD PER QUERY ROW (tcgen05.ld 32x32b hands each thread 32
@@ -15,10 +16,13 @@
 //              nears its capacity the warp re-tightens with a persistent 32-bin histogram of
 //              the buffered scores: the bin holding rank KEEP = k + max(m,1) is found, entries
 //              below it are dropped in place (stable, so entries stay in ascending chunk id)
-//              and the threshold moves to the smallest survivor.  After the last tile the cut
-//              at rank KEEP and the split at rank k are made exact inside their bins (directly
-//              for bins of up to 4 entries, else by zoom levels; a key-space radix level is
-//              the fallback for ranges too narrow to scale).  Ties go to the smaller chunk id.
+//              and the threshold moves to the smallest survivor.  After the last tile the bins
+//              of rank KEEP and rank k are located together on a second map laid over the
+//              stretch between them, the scores of those two bins are copied to short side
+//              lists and the exact ranks found there by counting; the cut is applied by the
+//              output pass.  Crowded bins, unusable ranges and wide bitmaps take the older
+//              way: top-2 / bottom-2 tracking, zoom levels, a key-space radix level for ranges
+//              too narrow to scale.  Ties go to the smaller chunk id.
 // Random sentinels are drawn by the same thread with the counter-based generator, using a
 // per-row bitmap of excluded chunks in shared memory.  Every mbarrier wait is bounded.
 #include "rr_common.cuh"

@@ -38,7 +38,7 @@ def oracle_params(w: W.RouteWorkload) -> O.OracleParams:
 
 
 def score_tol(qn: np.ndarray, kn_max: float, s_abs: np.ndarray) -> np.ndarray:
-    """fp32-accumulate error budget for a dot product of width d <= 128: the forward bound
+    """fp32-accumulate error allowance for a dot product of width d <= 128: the forward bound
     d * 2^-24 * |q|.|k| <= 7.7e-6 * ||q|| ||k||; we allow 1e-5 * ||q|| max||k|| + 1e-6 |s|.
     (The stated requirement, 1e-3 relative, is looser; it is asserted as well.)"""
     return 1e-5 * qn * kn_max + 1e-6 * np.abs(s_abs)
