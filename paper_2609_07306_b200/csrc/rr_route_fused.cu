@@ -33,7 +33,8 @@ using namespace sm100;
 namespace {
 
 constexpr int BM = 128, BN = 64, B_STAGES = 1, ACC_STAGES = 4, NT = 192;
-constexpr int TMEM_COLS = ACC_STAGES * BN;
+constexpr int A_COL = ACC_STAGES * BN;          // the Qc tile sits in TMEM behind the accumulators
+constexpr int TMEM_COLS = 512;                 // 4 x 64 accumulator columns + up to 64 of Qc, power of 2
 constexpr int NB = 32, NB_LOG = 5;             // histogram bins per level
 constexpr int CHUNK = 32;                      // scores handed to a thread per TMEM load
 constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -44,7 +45,7 @@ struct Cfg {
   static constexpr int A_BYTES = BM * D * 2, B_BYTES = BN * D * 2;
   static constexpr int A_HALF = BM * 128, B_HALF = BN * 128;   // rows x 128 bytes (64 bf16)
   static constexpr int CTL_BYTES = 2048;
-  static constexpr int FIXED_BYTES = 1024 + A_BYTES + B_STAGES * B_BYTES + CTL_BYTES;
+  static constexpr int FIXED_BYTES = 1024 + B_STAGES * B_BYTES + CTL_BYTES;
 };
 
 struct Ctl {
@@ -689,9 +690,8 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sA = smem;
-  uint8_t* sB = smem + C::A_BYTES;
-  Ctl* ctl = (Ctl*)(smem + C::A_BYTES + B_STAGES * C::B_BYTES);
+  uint8_t* sB = smem;
+  Ctl* ctl = (Ctl*)(smem + B_STAGES * C::B_BYTES);
   uint8_t* s_buf = (uint8_t*)ctl + C::CTL_BYTES;                      // [cap][BM] 8-byte entries
   uint8_t* s_aux = s_buf + (size_t)cap * ENTRY_PITCH;                 // [NB][BM] histogram words
 
@@ -726,29 +726,25 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   if (warp == 0) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
   __syncthreads();
 
-  // ---- gather the Qc tile into the K-major, 128B-swizzled layout -------------------------
-  {
-    constexpr int CPR = D / 8;
-    const __nv_bfloat16* qbase = qc + (size_t)prob * p.n_q * D;
-    // all of a thread's loads are issued before its first store: one memory round trip
-    constexpr int ITER = (BM * CPR + NT - 1) / NT;
-    uint4 vals[ITER];
+  // ---- the Qc tile goes to TMEM: the thread that owns row r loads the row (two bf16 per
+  // 32-bit word, as they lie in memory) and stores it to TMEM lane r, where the MMA reads its
+  // A operand from; rows without a query are zero
+  tc_fence_after();
+  if (warp >= 2) {
+    const int r = (warp & 3) * 32 + lane;
+    const int row = ctl->row[r];
+    constexpr int W = D / 2;                               // 32-bit words per row
+    uint32_t qv[W];
+    const uint4* src = reinterpret_cast<const uint4*>(qc + ((size_t)prob * p.n_q + max(row, 0)) * D);
 #pragma unroll
-    for (int i = 0; i < ITER; ++i) {
-      const int ch = tid + i * NT, r = ch / CPR, c16 = ch % CPR;
-      vals[i] = make_uint4(0, 0, 0, 0);
-      if (ch < BM * CPR) {
-        const int row = ctl->row[r];
-        if (row >= 0) vals[i] = __ldg(reinterpret_cast<const uint4*>(qbase + (size_t)row * D + c16 * 8));
-      }
+    for (int i = 0; i < W / 4; ++i) {
+      uint4 t = make_uint4(0, 0, 0, 0);
+      if (row >= 0) t = __ldg(src + i);
+      qv[4 * i] = t.x; qv[4 * i + 1] = t.y; qv[4 * i + 2] = t.z; qv[4 * i + 3] = t.w;
     }
-#pragma unroll
-    for (int i = 0; i < ITER; ++i) {
-      const int ch = tid + i * NT, r = ch / CPR, c16 = ch % CPR, h = c16 >> 3, cc = c16 & 7;
-      if (ch < BM * CPR)
-        *reinterpret_cast<uint4*>(sA + h * C::A_HALF + r * 128 + ((cc ^ (r & 7)) << 4)) = vals[i];
-    }
-    fence_proxy_async_smem();
+    const uint32_t taddr = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_COL;
+    if constexpr (W == 64) tmem_st_32x64(taddr, qv); else tmem_st_32x32(taddr, qv);
+    tmem_st_wait();
   }
   tc_fence_before();
   __syncthreads();
@@ -784,7 +780,6 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     // ===== MMA issuer =====
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
-      const uint32_t a_addr = smem_u32(sA);
       for (int t = 0; t < n_tiles; ++t) {
         const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
         const int as = t % ACC_STAGES; const uint32_t aph = (t / ACC_STAGES) & 1;
@@ -794,10 +789,9 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         const uint32_t b_addr = smem_u32(sB + s * C::B_BYTES);
 #pragma unroll
         for (int k = 0; k < C::KSTEPS; ++k) {
-          const uint32_t a_off = (k >> 2) * C::A_HALF + (k & 3) * 32;
           const uint32_t b_off = (k >> 2) * C::B_HALF + (k & 3) * 32;
-          umma_bf16(tmem_base + as * BN, umma_desc_k_sw128(a_addr + a_off),
-                    umma_desc_k_sw128(b_addr + b_off), idesc, k > 0 ? 1u : 0u);
+          umma_bf16_ts(tmem_base + as * BN, tmem_base + A_COL + k * 8,
+                       umma_desc_k_sw128(b_addr + b_off), idesc, k > 0 ? 1u : 0u);
         }
         umma_commit(&ctl->empty[s]);
         umma_commit(&ctl->acc_full[as]);
@@ -1072,7 +1066,7 @@ bool plan(const RRParams& p, int& cap, int& aux_words, size_t& smem_bytes) {
   const size_t hist = (size_t)NB * AUX_PITCH;
   if (fixed + hist >= max_smem) return false;
   const int fit = (int)((max_smem - fixed - hist) / ENTRY_PITCH);
-  cap = keep + 112;
+  cap = keep + 144;
   if (cap > fit) cap = fit;
   if (cap < keep + CHUNK) return false;
   // a bitmap wider than the histogram lives in the buffer entries beyond `keep`
