@@ -93,6 +93,9 @@ typedef struct rr_config {
   float   gamma_boost;     /* hysteresis: added to gamma for rows whose margin (Section 3.3)
                               recorded at their last routing is below margin_recover        */
   float   margin_recover;
+  int32_t coalesce_ranges; /* with chunk_tokens > 0: runs of consecutive selected chunks become
+                              one token range (the form a sparse-attention kernel consumes);
+                              a row then holds its merged ranges first, (-1,-1) after them  */
 } rr_config;
 
 /* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */

@@ -450,14 +450,20 @@ def run_layers(q_layers: np.ndarray, k_layers: np.ndarray, p: OracleParams,
     return results, summary
 
 
-def token_ranges(routes: np.ndarray, chunk_tokens: int) -> np.ndarray:
+def token_ranges(routes: np.ndarray, chunk_tokens: int, coalesce: bool = False) -> np.ndarray:
     """Expansion of selected chunks into token index ranges (Sec 2.1): each row's chunk ids
-    in ascending order, chunk j -> [j*T, (j+1)*T); empty slots (-1,-1) at the end."""
+    in ascending order, chunk j -> [j*T, (j+1)*T); empty slots (-1,-1) at the end.
+    With `coalesce`, runs of consecutive chunk ids become one range."""
     rows, k = routes.shape
     out = np.full((rows, k, 2), -1, np.int32)
     for i in range(rows):
         ids = sorted(int(j) for j in routes[i] if j >= 0)
-        for s, j in enumerate(ids):
+        s = 0
+        for pos, j in enumerate(ids):
+            if coalesce and pos > 0 and ids[pos - 1] == j - 1:
+                out[i, s - 1, 1] = (j + 1) * chunk_tokens       # extends the current run
+                continue
             out[i, s, 0] = j * chunk_tokens
             out[i, s, 1] = (j + 1) * chunk_tokens
+            s += 1
     return out

@@ -39,7 +39,8 @@ class rr_config(C.Structure):
                 ("causal_offset", C.c_int32), ("gamma", C.c_float), ("seed", C.c_uint64),
                 ("chunk_tokens", C.c_int32), ("debug_outputs", C.c_int32),
                 ("global_sentinels", C.c_int32), ("min_reuse", C.c_int32), ("h_max", C.c_int32),
-                ("gamma_boost", C.c_float), ("margin_recover", C.c_float)]
+                ("gamma_boost", C.c_float), ("margin_recover", C.c_float),
+                ("coalesce_ranges", C.c_int32)]
 
 
 class rr_views(C.Structure):

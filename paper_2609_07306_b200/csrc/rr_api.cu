@@ -49,6 +49,7 @@ int validate(const rr_config* c) {
   if (c->global_sentinels < 0 || c->global_sentinels > 3) return RR_ERR_INVALID_ARG;
   if (c->min_reuse < 0 || c->h_max < 0 || !(c->gamma_boost >= 0.f)) return RR_ERR_INVALID_ARG;
   if (c->margin_recover != c->margin_recover) return RR_ERR_INVALID_ARG;   // NaN
+  if (c->coalesce_ranges != 0 && c->coalesce_ranges != 1) return RR_ERR_INVALID_ARG;
   if (c->k + c->m + c->r + (c->global_sentinels & 1) + ((c->global_sentinels >> 1) & 1) > RR_MAX_C)
     return RR_ERR_UNSUPPORTED;
   const long long rows = (long long)c->batch * c->heads * c->n_q;
@@ -70,6 +71,7 @@ RRParams shape_params(const rr_config* cfg) {
   p.sw = cfg->m + cfg->r + p.n_global; p.c = cfg->k + p.sw;
   p.dtype = cfg->dtype; p.causal = cfg->causal; p.causal_offset = cfg->causal_offset;
   p.chunk_tokens = cfg->chunk_tokens; p.debug = cfg->debug_outputs & 1;
+  p.coalesce = cfg->coalesce_ranges;
   p.rows = p.P * p.n_q;
   p.tiles_per_problem = (p.n_q + RR_ROW_TILE - 1) / RR_ROW_TILE;
   p.n_tiles = p.P * p.tiles_per_problem;

@@ -16,6 +16,7 @@ struct RRParams {
   int global_mask, n_global, min_reuse, h_max;   // optional policies (0 = off)
   float gamma_boost, margin_recover;
   int dtype, causal, causal_offset, chunk_tokens, debug;   // debug: bit 0 = store candidate scores
+  int coalesce;                            // token ranges of adjacent chunks merged
   int rows, tiles_per_problem, n_tiles;    // row tiles of RR_ROW_TILE per problem / in total
   float gamma;
   unsigned long long seed;

@@ -106,7 +106,42 @@ expand_kernel(RRParams p, int is_anchor) {
     const int id = route[s];
     if (s > 0 && id >= 0) { const int prev = route[s - 1]; ordered &= prev >= 0 && prev < id; }
   }
-  if (__all_sync(FULL, ordered)) {
+  const bool all_ordered = __all_sync(FULL, ordered);
+  if (p.coalesce) {
+    // the row's ids in ascending order (empty slots last) into shared memory, then one range
+    // per run of consecutive ids: a run's first id writes its start, its last id its end
+    extern __shared__ int32_t s_sorted[];
+    int32_t* srt = s_sorted + (threadIdx.x >> 5) * p.k;
+    for (int s = lane; s < p.k; s += 32) srt[s] = all_ordered ? route[s] : -1;
+    __syncwarp();
+    if (!all_ordered) {
+      for (int s = lane; s < p.k; s += 32) {
+        const int id = route[s];
+        if (id >= 0) {
+          int rank = 0;
+          for (int t = 0; t < p.k; ++t) { const int o = route[t]; rank += (o >= 0 && o < id); }
+          srt[rank] = id;
+        }
+      }
+      __syncwarp();
+    }
+    int base = 0;
+    for (int s0 = 0; s0 < p.k; s0 += 32) {
+      const int s = s0 + lane;
+      const int id = s < p.k ? srt[s] : -1;
+      const bool valid = id >= 0;
+      const bool joins_prev = valid && s > 0 && srt[s - 1] == id - 1 && srt[s - 1] >= 0;
+      const bool joins_next = valid && s + 1 < p.k && srt[s + 1] == id + 1;
+      const unsigned starts = __ballot_sync(FULL, valid && !joins_prev);
+      const int ri = base + __popc(starts & (0xFFFFFFFFu >> (31 - lane))) - 1;
+      if (valid && !joins_prev) out[2 * ri] = id * p.chunk_tokens;
+      if (valid && !joins_next) out[2 * ri + 1] = (id + 1) * p.chunk_tokens;
+      base += __popc(starts);
+    }
+    for (int s = base + lane; s < p.k; s += 32) { out[2 * s] = -1; out[2 * s + 1] = -1; }
+    return;
+  }
+  if (all_ordered) {
     for (int s = lane; s < p.k; s += 32) {
       const int id = route[s];
       reinterpret_cast<int2*>(out)[s] =
@@ -168,7 +203,8 @@ cudaError_t rr_launch_update(const RRParams& p, int is_anchor, unsigned long lon
   rr_count_launch();
   if (p.chunk_tokens > 0) {
     const int wpb = 8;
-    expand_kernel<<<(p.rows + wpb - 1) / wpb, wpb * 32, 0, st>>>(p, is_anchor);
+    const size_t smem = p.coalesce ? (size_t)wpb * p.k * sizeof(int32_t) : 0;
+    expand_kernel<<<(p.rows + wpb - 1) / wpb, wpb * 32, smem, st>>>(p, is_anchor);
     rr_count_launch();
   }
   return cudaPeekAtLastError();

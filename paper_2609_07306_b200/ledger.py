@@ -22,7 +22,8 @@ def config_from_workload(w: RouteWorkload, debug_outputs: bool = False,
                        (4 if gathered else 0),
                        global_sentinels=int(w.global_sentinels), min_reuse=int(w.min_reuse),
                        h_max=int(w.h_max), gamma_boost=float(w.gamma_boost),
-                       margin_recover=float(w.margin_recover))
+                       margin_recover=float(w.margin_recover),
+                       coalesce_ranges=1 if w.coalesce_ranges else 0)
 
 
 class RouteLedger:

@@ -59,6 +59,7 @@ class RouteWorkload:
     redraw_every: int = 0     # 0 = never
     redraw_frac: float = 0.0
     chunk_tokens: int = 0     # >0: routes are also expanded to token ranges
+    coalesce_ranges: bool = False   # token ranges of adjacent chunks merged
     causal_offset: int = 0    # causal: row i sees chunks j < min(n_k, i + 1 + causal_offset)
     # optional policies (Section 3.1 item 3, Section 3.2 "Hysteresis" / "Forced anchors")
     global_sentinels: int = 0   # bit 0: sink chunk, bit 1: most recent chunk

@@ -194,15 +194,23 @@ def test_pipelined_host_layers_entry_point():
     led.close(); ref.close()
 
 
-def test_token_ranges():
-    w = W.moderate().replace(heads=2, chunk_tokens=64)
+@pytest.mark.parametrize("coalesce", [False, True], ids=["per_chunk", "coalesced"])
+@pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
+def test_token_ranges(two_pass, coalesce):
+    """Token ranges of the routes (per chunk, or runs of adjacent chunks merged), from rows in
+    ascending chunk id (fused kernel) and in rank order (two-pass path, imported ledgers)."""
+    w = W.moderate().replace(heads=2, chunk_tokens=64, coalesce_ranges=coalesce)
     q, k = W.generate(w, layers=2)
-    led = RouteLedger(config_from_workload(w))
+    led = RouteLedger(config_from_workload(w, two_pass=two_pass))
     led.route_anchor(device_tensor(q[0]), device_tensor(k[0]), 0)
     led.route_relay(device_tensor(q[1]), device_tensor(k[1]), 1)
     torch.cuda.synchronize()
-    expect = O.token_ranges(led.routes.cpu().numpy(), 64)
+    routes = led.routes.cpu().numpy()
+    expect = O.token_ranges(routes, 64, coalesce=coalesce)
     assert np.array_equal(led.token_ranges.cpu().numpy(), expect)
+    if coalesce:      # the causal rows select runs of neighbours: something must have merged
+        per_chunk = O.token_ranges(routes, 64)
+        assert (expect[:, :, 0] >= 0).sum() < (per_chunk[:, :, 0] >= 0).sum()
     led.close()
 
 

@@ -344,6 +344,12 @@ def test_token_ranges():
     tr = O.token_ranges(routes, 64)
     assert tr[0].tolist() == [[128, 192], [320, 384], [-1, -1]]
     assert tr[1].tolist() == [[0, 64], [192, 256], [448, 512]]
+    # coalesced: runs of consecutive chunks merge (hand-worked: {3,4,5}, {9}, {11,12}, T = 10)
+    routes = np.array([[12, 3, 9, 5, 4, 11, -1]], np.int32)
+    tr = O.token_ranges(routes, 10, coalesce=True)
+    assert tr[0].tolist() == [[30, 60], [90, 100], [110, 130], [-1, -1], [-1, -1], [-1, -1], [-1, -1]]
+    assert O.token_ranges(routes, 10)[0, :6].tolist() == [[30, 40], [40, 50], [50, 60], [90, 100],
+                                                         [110, 120], [120, 130]]
 
 
 def test_relay_requires_anchor():
