@@ -4,7 +4,7 @@
 // the FP32 ALUs: no operand is reused, so it moves c*d*2 bytes per row through L2 and is an
 // order of magnitude slower on this machine than computing the whole score strip with
 // tcgen05.mma.  This variant does the latter: the same kind of tile pipeline as the fused
-// routing kernel produces S[128 rows, 32 chunks] tiles in TMEM, and the threads of a row pick
+// routing kernel produces S[128 rows, 64 chunks] tiles in TMEM, and the threads of a row pick
 // out the scores of the row's candidates:
 //   * at start the two threads of a row turn its ledger row into a bitmap in shared memory (two
 //     planes encoding route / near-miss / random sentinel, one plane per thread), reading the
@@ -24,11 +24,11 @@ using namespace sm100;
 
 namespace {
 
-// 32-chunk tiles keep a CTA under half an SM's shared memory: two CTAs per SM overlap one's
-// set-up and bitmap build with the other's tile loop.  Two threads share a query row (each
-// takes 16 of a tile's 32 columns): the per-tile work is a chain of dependent ALU-pipe
+// 64-chunk tiles in two stages keep a CTA under half an SM's shared memory: two CTAs per SM
+// overlap one's set-up and bitmap build with the other's tile loop.  Two threads share a query
+// row (each takes 32 of a tile's 64 columns, one bitmap word): the per-tile work is a chain of dependent ALU-pipe
 // instructions, so twice the warps hide twice the latency.
-constexpr int BN = 32, B_STAGES = 3, ACC_STAGES = 4;
+constexpr int BN = 64, B_STAGES = 2, ACC_STAGES = 4;
 constexpr int TPR = 2, COLS = BN / TPR;             // threads per row, columns per thread
 constexpr int NCONS = tcpipe::BM * TPR, NT = 64 + NCONS;
 constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -208,14 +208,15 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
       // after a wait that gave up the remaining iterations only keep the barriers in step
       if (alive) alive = pipe.consumer_wait(t);
       RD_LAP(2);
-      static_assert(BN == 32, "a tile is one bitmap word");
-      const bool in = alive && t < words;
-      const uint32_t wa = in ? lds(bA + t * 4u) >> sh : 0u, wb = in ? lds(bB + t * 4u) >> sh : 0u;
+      static_assert(COLS == 32, "a thread's share of a tile is one bitmap word");
+      const int wi = t * TPR + part;                       // this thread's word of either plane
+      const bool in = alive && wi < words;
+      const uint32_t wa = in ? lds(bA + wi * 4u) : 0u, wb = in ? lds(bB + wi * 4u) : 0u;
       const uint32_t wr = wa & ~wb, wn = wb & ~wa, ws = wb;
-      const bool work = __any_sync(FULL, ((wa | wb) & ((1u << COLS) - 1u)) != 0u);
+      const bool work = __any_sync(FULL, (wa | wb) != 0u);
       uint32_t a0[COLS];
       if (work) {
-        tmem_ld_32x16(pipe.acc_addr(t, quarter) + sh, a0);
+        tmem_ld_32x32(pipe.acc_addr(t, quarter) + sh, a0);
         // masked min / max straight from the registers: no loop over set bits (its trip
         // count and its dependent shared-memory reads made it several times slower)
 #pragma unroll
