@@ -143,7 +143,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   } while (0)
   if (anchor) {
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
-    LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, st));
+    LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, L->dense_pairs_per_layer, st));
     if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, nullptr, layer, st));
     } else {
@@ -151,14 +151,13 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
       else LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, nullptr, st));
       LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, nullptr, layer, st));
     }
-    LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 1, L->dense_pairs_per_layer, st));
     L->anchored = 1;
   } else {
     if (!L->anchored) return RR_ERR_STATE;
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
     if (L->dense_rescore) LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, st));
     else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
-    LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, st));
+    LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
     if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
     } else {
@@ -168,8 +167,8 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
         LAUNCH(RR_KIND_SCORE_SIMT, rr_launch_score_simt(p, qc, kc, p.refresh_rows, st));
       LAUNCH(RR_KIND_TOPK_ROWS, rr_launch_topk_rows(p, p.refresh_rows, layer, st));
     }
-    LAUNCH(RR_KIND_UPDATE, rr_launch_update(p, 0, L->dense_pairs_per_layer, st));
   }
+  if (p.chunk_tokens > 0) LAUNCH(RR_KIND_EXPAND, rr_launch_expand(p, anchor ? 1 : 0, st));
 #undef LAUNCH
   return RR_OK;
 }

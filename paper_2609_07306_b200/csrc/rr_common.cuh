@@ -116,10 +116,11 @@ cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
 bool rr_rescore_dense_supported(const RRParams& p);
 cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
                                     cudaStream_t st);
-cudaError_t rr_launch_compact(const RRParams& p, cudaStream_t st);
-cudaError_t rr_launch_anchor_fill(const RRParams& p, cudaStream_t st);
-cudaError_t rr_launch_update(const RRParams& p, int is_anchor, unsigned long long dense_pairs,
-                             cudaStream_t st);
+// compact / anchor_fill also advance the ages and the cumulative counters of the layer
+cudaError_t rr_launch_compact(const RRParams& p, unsigned long long dense_pairs, cudaStream_t st);
+cudaError_t rr_launch_anchor_fill(const RRParams& p, unsigned long long dense_pairs,
+                                  cudaStream_t st);
+cudaError_t rr_launch_expand(const RRParams& p, int is_anchor, cudaStream_t st);
 cudaError_t rr_launch_reset(const RRParams& p, cudaStream_t st);
 
 void rr_count_launch(int n = 1);

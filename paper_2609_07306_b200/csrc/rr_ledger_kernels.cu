@@ -1,6 +1,7 @@
-// Row compaction (Section 4.2: "A prefix sum compacts unstable row IDs"), the ledger-update
-// kernel (Section 4.1: stable rows keep their routes and their ages advance; refreshed rows
-// restart at age 0), token-range expansion, and ledger reset.
+// Row compaction (Section 4.2: "A prefix sum compacts unstable row IDs") together with the
+// ledger's book-keeping (Section 4.1: stable rows keep their routes and their ages advance;
+// refreshed rows restart at age 0; cumulative work counters), the anchor's fill of the same
+// state, token-range expansion, and ledger reset.
 #include "rr_common.cuh"
 
 namespace {
@@ -12,8 +13,10 @@ constexpr unsigned FULL = 0xFFFFFFFFu;
 // of the flagged counts of all earlier tiles (written by the rescoring kernel); inside the
 // tile a ballot/popcount scan gives each flagged row its slot.  The list is therefore in
 // ascending global row id -- exactly numpy.nonzero(flags) -- with no atomics and no waits.
+// The same pass advances the ages (flagged -> 0, stable -> +1) and, once per launch, the
+// per-layer counters: nothing later in the layer reads either.
 __global__ void __launch_bounds__(RR_ROW_TILE)
-compact_kernel(RRParams p) {
+compact_kernel(RRParams p, unsigned long long dense_pairs) {
   __shared__ int s_part[RR_ROW_TILE / 32];
   __shared__ int s_base;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -44,7 +47,13 @@ compact_kernel(RRParams p) {
   int before = 0;
   for (int w = 0; w < warp; ++w) before += s_part[w];
   if (f) p.refresh_rows[base + before + __popc(bal & ((1u << lane) - 1u))] = g;
+  if (i < p.n_q) p.ages[g] = f ? 0 : p.ages[g] + 1;
   if (tid == 0) {
+    if (tile_id == 0) {
+      p.counters[RR_CNT_LAYER_CALLS] += 1;
+      p.counters[RR_CNT_DENSE_PAIRS] += dense_pairs;
+      p.counters[RR_CNT_RELAY_ROWS] += (unsigned long long)p.rows;
+    }
     if (tile == 0) p.problem_offsets[prob] = base;
     if (tile_id == p.n_tiles - 1) {
       int total = base;
@@ -56,7 +65,8 @@ compact_kernel(RRParams p) {
 }
 
 // ---- anchor: every row is (re)routed ----------------------------------------------------
-__global__ void anchor_fill_kernel(RRParams p) {
+// Flags, identity refresh list, offsets, ages and the anchor's counters.
+__global__ void anchor_fill_kernel(RRParams p, unsigned long long dense_pairs) {
   const int g = blockIdx.x * blockDim.x + threadIdx.x;
   const float qnan = __int_as_float(0x7fc00000);
   if (g < p.rows) {
@@ -64,33 +74,21 @@ __global__ void anchor_fill_kernel(RRParams p) {
     p.refresh_rows[g] = g;
     p.alpha[g] = qnan;
     p.beta[g] = qnan;
+    p.ages[g] = 0;
   }
   if (g <= p.P) p.problem_offsets[g] = g * p.n_q;
-  if (g == 0) *p.refresh_count = p.rows;
-}
-
-// ---- ledger update ------------------------------------------------------------------------
-// Ages, cumulative work counters and (optionally) the token ranges of the rows that were
-// re-routed.  One warp per row for the expansion: ids are ranked by counting (they are
-// distinct), chunk j -> [j*T, (j+1)*T), ascending chunk id, (-1,-1) for empty slots.
-__global__ void __launch_bounds__(256)
-update_kernel(RRParams p, int is_anchor, unsigned long long dense_pairs) {
-  const int g = blockIdx.x * blockDim.x + threadIdx.x;
   if (g == 0) {
+    *p.refresh_count = p.rows;
     p.counters[RR_CNT_LAYER_CALLS] += 1;
     p.counters[RR_CNT_DENSE_PAIRS] += dense_pairs;
-    if (is_anchor) {
-      p.counters[RR_CNT_ANCHOR_ROWS] += (unsigned long long)p.rows;
-      p.counters[RR_CNT_FULL_PAIRS] += dense_pairs;
-    } else {
-      p.counters[RR_CNT_RELAY_ROWS] += (unsigned long long)p.rows;
-    }
+    p.counters[RR_CNT_ANCHOR_ROWS] += (unsigned long long)p.rows;
+    p.counters[RR_CNT_FULL_PAIRS] += dense_pairs;
   }
-  if (g >= p.rows) return;
-  const bool refreshed = is_anchor || p.flags[g] != 0;
-  p.ages[g] = refreshed ? 0 : p.ages[g] + 1;
 }
 
+// ---- token ranges of the rows that were re-routed -------------------------------------------
+// One warp per row: ids are ranked by counting (they are distinct), chunk j -> [j*T, (j+1)*T),
+// ascending chunk id, (-1,-1) for empty slots.
 __global__ void __launch_bounds__(256)
 expand_kernel(RRParams p, int is_anchor) {
   const int lane = threadIdx.x & 31;
@@ -184,29 +182,25 @@ __global__ void reset_kernel(RRParams p) {
 
 }  // namespace
 
-cudaError_t rr_launch_compact(const RRParams& p, cudaStream_t st) {
-  compact_kernel<<<p.n_tiles, RR_ROW_TILE, 0, st>>>(p);
+cudaError_t rr_launch_compact(const RRParams& p, unsigned long long dense_pairs, cudaStream_t st) {
+  compact_kernel<<<p.n_tiles, RR_ROW_TILE, 0, st>>>(p, dense_pairs);
   rr_count_launch();
   return cudaPeekAtLastError();
 }
 
-cudaError_t rr_launch_anchor_fill(const RRParams& p, cudaStream_t st) {
+cudaError_t rr_launch_anchor_fill(const RRParams& p, unsigned long long dense_pairs,
+                                  cudaStream_t st) {
   const int n = p.rows > p.P + 1 ? p.rows : p.P + 1;
-  anchor_fill_kernel<<<(n + 255) / 256, 256, 0, st>>>(p);
+  anchor_fill_kernel<<<(n + 255) / 256, 256, 0, st>>>(p, dense_pairs);
   rr_count_launch();
   return cudaPeekAtLastError();
 }
 
-cudaError_t rr_launch_update(const RRParams& p, int is_anchor, unsigned long long dense_pairs,
-                             cudaStream_t st) {
-  update_kernel<<<(p.rows + 255) / 256, 256, 0, st>>>(p, is_anchor, dense_pairs);
+cudaError_t rr_launch_expand(const RRParams& p, int is_anchor, cudaStream_t st) {
+  const int wpb = 8;
+  const size_t smem = p.coalesce ? (size_t)wpb * p.k * sizeof(int32_t) : 0;
+  expand_kernel<<<(p.rows + wpb - 1) / wpb, wpb * 32, smem, st>>>(p, is_anchor);
   rr_count_launch();
-  if (p.chunk_tokens > 0) {
-    const int wpb = 8;
-    const size_t smem = p.coalesce ? (size_t)wpb * p.k * sizeof(int32_t) : 0;
-    expand_kernel<<<(p.rows + wpb - 1) / wpb, wpb * 32, smem, st>>>(p, is_anchor);
-    rr_count_launch();
-  }
   return cudaPeekAtLastError();
 }
 
