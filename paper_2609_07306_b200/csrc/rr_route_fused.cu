@@ -763,7 +763,7 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       int issued = 0;
       for (int t = 0; t < n_tiles; ++t) {
         const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
-        if (!mbar_wait(&ctl->empty[s], ph ^ 1, abort_flag)) break;
+        if (!mbar_wait_relaxed(&ctl->empty[s], ph ^ 1, abort_flag, 400)) break;
         mbar_expect_tx(&ctl->full[s], C::B_BYTES);
 #pragma unroll
         for (int h = 0; h < C::KHALVES; ++h)
@@ -783,8 +783,8 @@ route_fused_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       for (int t = 0; t < n_tiles; ++t) {
         const int s = t % B_STAGES; const uint32_t ph = (t / B_STAGES) & 1;
         const int as = t % ACC_STAGES; const uint32_t aph = (t / ACC_STAGES) & 1;
-        if (!mbar_wait(&ctl->acc_empty[as], aph ^ 1, abort_flag)) break;
-        if (!mbar_wait(&ctl->full[s], ph, abort_flag)) break;
+        if (!mbar_wait_relaxed(&ctl->acc_empty[as], aph ^ 1, abort_flag, 400)) break;
+        if (!mbar_wait_relaxed(&ctl->full[s], ph, abort_flag, 100)) break;
         tc_fence_after();
         const uint32_t b_addr = smem_u32(sB + s * C::B_BYTES);
 #pragma unroll

@@ -53,6 +53,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   *abort_flag = 1u;
   return false;
 }
+// The same for the roles that run far ahead of the consumers (the TMA producer and the MMA
+// issuer): they sleep between polls from the first miss on, so that their polling does not take
+// issue slots from the warps that share their schedulers.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity,
+                                                  volatile uint32_t* abort_flag, uint32_t ns) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    __nanosleep(ns);
+  }
+  *abort_flag = 1u;
+  return false;
+}
 
 // ---- proxies / fences -----------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
