@@ -155,8 +155,8 @@ class ClockSampler:
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels that
 # dominate a high_drift step, from the ncu captures summarised in profiles/
 # (route_fused_high_drift.md: 199.2 MB anchor / 204.3 MB refresh; rescore_dense_high_drift.md).
-NCU_TRAFFIC_BYTES = {"high_drift": {"route_fused": (4 * 197.5e6 + 28 * 200.8e6) / 32,
-                                    "rescore_dense": 241.0e6}}
+NCU_TRAFFIC_BYTES = {"high_drift": {"route_fused": (4 * 199.3e6 + 28 * 200.6e6) / 32,
+                                    "rescore_dense": 244.2e6}}
 
 
 # ----------------------------------------------------------------------------- roofline
