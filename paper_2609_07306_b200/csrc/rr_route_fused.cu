@@ -491,6 +491,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
   const int from = usable ? st.binned : 0, to = usable ? n : 0;
   const int nw_new = warp_max(to - from);
   float mlo = st.map_lo, msc = st.map_scale;
+  float moff = -mlo * msc;           // bin coordinate of a score: fmaf(v, msc, moff), everywhere
   for (int e0 = 0; e0 < nw_new; e0 += BATCH) {
     float v[BATCH];
 #pragma unroll
@@ -500,7 +501,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
       inc[j] = from + e0 + j < to ? 1u : 0u;
-      b[j] = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+      b[j] = max(0, min(NB - 1, __float2int_rz(fmaf(v[j], msc, moff))));
     }
     hist_add(s.aux, b, inc);
   }
@@ -523,7 +524,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       const float e_lo = mlo + (float)bsel / msc, e_hi = mlo + (float)(bsel_k + 1) / msc;
       const float w = (e_hi - e_lo) * (1.0f / (float)(NB - 2));
       const bool remap = usable && w > 0.f && (1.0f / w) < 1e37f;
-      if (remap) { mlo = e_lo - w; msc = 1.0f / w; }
+      if (remap) { mlo = e_lo - w; msc = 1.0f / w; moff = -mlo * msc; }
       clear_bins_if(remap, s);
       const int nr_ = remap ? n : 0;
       for (int e0 = 0; e0 < nw; e0 += BATCH) {
@@ -534,7 +535,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
           inc[j] = e0 + j < nr_ ? 1u : 0u;
-          b[j] = max(0, min(NB - 1, __float2int_rz((v[j] - mlo) * msc)));
+          b[j] = max(0, min(NB - 1, __float2int_rz(fmaf(v[j], msc, moff))));
         }
         hist_add(s.aux, b, inc);
       }
@@ -567,7 +568,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
         ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
 #pragma unroll
       for (int j = 0; j < BATCH; ++j) {
-        const float t = (v[j] - mlo) * msc;
+        const float t = fmaf(v[j], msc, moff);
         const bool live = e0 + j < nd;
         const bool keep_it = live & (t >= tb);
         const int b = max(0, min(NB - 1, __float2int_rz(t)));
@@ -598,7 +599,7 @@ __device__ void retighten(const Sel& s, bool active, int& n, int keep, int fit_l
       ld_entry(s.buf + min(e0 + j, max(nd - 1, 0)) * ENTRY_PITCH, v[j], id[j]);
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
-      const float t = (v[j] - mlo) * msc;
+      const float t = fmaf(v[j], msc, moff);
       const bool live = e0 + j < nd;
       const bool keep_it = live & (t >= tb);
       if (FINAL) {
