@@ -240,7 +240,7 @@ int rr_compact_flags_noalloc(const uint8_t* dev_flags, int32_t n_problems, int32
 #define RR_KIND_RESCORE      2   /* gathered candidate rescoring + challenge test            */
 #define RR_KIND_COMPACT      3   /* ballot / prefix-scan row compaction + ages and counters  */
 #define RR_KIND_ANCHOR_FILL  4   /* anchor: flags, identity refresh list, ages, counters     */
-#define RR_KIND_UPDATE       5   /* (not launched any more: folded into kinds 3 and 4)       */
+#define RR_KIND_UPDATE       5   /* reserved: ages and counters are written by kinds 3 and 4  */
 #define RR_KIND_EXPAND       6   /* token-range expansion                                    */
 #define RR_KIND_SCORE_TC     7   /* tcgen05 score GEMM                                       */
 #define RR_KIND_ROUTE_FUSED  8   /* tcgen05 score GEMM fused with TopK + sentinels           */
