@@ -124,3 +124,13 @@ cudaError_t rr_launch_expand(const RRParams& p, int is_anchor, cudaStream_t st);
 cudaError_t rr_launch_reset(const RRParams& p, cudaStream_t st);
 
 void rr_count_launch(int n = 1);
+
+// Function attributes (dynamic shared-memory limit) are per device: true the first time the
+// calling site runs on the current device.  `done` is the site's own bit mask of devices.
+inline bool rr_first_use_on_device(unsigned long long& done) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev > 63) return true;
+  if ((done >> dev) & 1ull) return false;
+  done |= 1ull << dev;
+  return true;
+}

@@ -319,8 +319,8 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
   if (e != cudaSuccess) return e;
   e = rr_encode_tmap_bf16_3d(&tmap_q, qc, p.d, p.n_q, p.P, tcpipe::BM);
   if (e != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_done = 0;      // devices on which the attributes are set
+  if (rr_first_use_on_device(attr_done)) {
     e = cudaFuncSetAttribute(rescore_dense_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              227 * 1024);
     if (e != cudaSuccess) return e;
@@ -329,7 +329,6 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
     if (e != cudaSuccess) return e;
     cudaFuncSetAttribute(rescore_dense_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    attr_set = true;
   }
   const int grid = p.n_tiles;
   if (p.d == 128)

@@ -1113,15 +1113,14 @@ cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void*
   const int grid = p.P * p.tiles_per_problem;
   const int keep = p.k + (p.m > 0 ? p.m : 1);
   const bool fine = cap - keep < 64;             // little room above keep: check the fill more often
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_done = 0;      // devices on which the attributes are set
+  if (rr_first_use_on_device(attr_done)) {
     const void* fns[4] = {(const void*)route_fused_kernel<128, 32>, (const void*)route_fused_kernel<128, 8>,
                           (const void*)route_fused_kernel<64, 32>, (const void*)route_fused_kernel<64, 8>};
     for (const void* fn : fns) {
       e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
       if (e != cudaSuccess) return e;
     }
-    attr_set = true;
   }
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   if (p.d == 128 && !fine)

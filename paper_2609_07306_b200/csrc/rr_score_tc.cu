@@ -226,15 +226,14 @@ cudaError_t rr_launch_score_tc(const RRParams& p, const void* qc, const void* kc
   cudaError_t e = rr_encode_tmap_bf16_3d(&tmap, kc, p.d, p.n_k, p.P, BN);
   if (e != cudaSuccess) return e;
   const int grid = p.P * p.tiles_per_problem;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_done = 0;      // devices on which the attributes are set
+  if (rr_first_use_on_device(attr_done)) {
     e = cudaFuncSetAttribute(score_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg<128>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(score_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg<64>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   if (p.d == 128)
     score_tc_kernel<128><<<grid, NT, Cfg<128>::SMEM_BYTES, st>>>(p, (const __nv_bfloat16*)qc, tmap,
