@@ -499,8 +499,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="high_drift",
-                    help="one of %s, or sweep_<n>_<rho> (BASELINE configuration 3, e.g. "
-                         "sweep_256_0.15)" % ", ".join(sorted(W.PRESETS) + ["sweep1024"]))
+                    help="one of %s, or sweep_<n>_<rho> (the routing-scale sweep: 32 heads, n "
+                         "chunks, drift rho; e.g. sweep_256_0.15)"
+                         % ", ".join(sorted(W.PRESETS) + ["sweep1024"]))
     ap.add_argument("--graph", action="store_true",
                     help="time the device-resident step as replays of one CUDA graph of it "
                          "(for the launch-bound small shapes)")

@@ -129,7 +129,9 @@ typedef struct rr_views {
 #define RR_CNT_DENSE_PAIRS   6   /* what full routing on every layer would have scored        */
 #define RR_NUM_COUNTERS      8
 
-/* Sizes of the two caller-owned device buffers for a configuration.  Host-only. */
+/* Sizes of the two caller-owned device buffers for a configuration (Section 4.4: the ledger is
+ * rows * (k + m + r) 32-bit indices plus a few words per row; the scratch holds the per-layer
+ * flags, alpha / beta, the refresh list and counters).  Host-only. */
 int rr_workspace_bytes(const rr_config* cfg, size_t* ledger_bytes, size_t* scratch_bytes);
 
 /* Creates the host handle over caller-owned device buffers (both 256-byte aligned, at least
@@ -171,8 +173,12 @@ int rr_route_layer_host(rr_ledger* L, const void* host_qc, const void* host_kc,
  *   host_routes         [n_layers] host pointers (rows*k int32 each) or NULL entries / NULL
  *   d2h_stream          stream of the route downloads (NULL = copy_stream); a separate one lets
  *                       uploads and downloads use both directions of the link at once
- * Enqueue-only: the caller synchronises ALL streams before reading host_routes or reusing
- * any buffer.  The library creates a few CUDA events on first use (no device memory). */
+ * Enqueue-only: the caller synchronises ALL streams before reading host_routes or touching a
+ * buffer itself.  Calls on the same ledger with the same staging buffers may follow one
+ * another without a synchronisation in between: the library orders each reuse of a staging
+ * set behind its previous reader (events kept in the ledger; a few are created on first use,
+ * no device memory).  host_routes entries must not repeat while a download may still be in
+ * flight. */
 int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host_qc,
                          const void* const* host_kc, const int32_t* is_anchor,
                          int32_t first_layer, void* const* dev_qc_staging,
@@ -183,8 +189,9 @@ int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host
 /* Device pointers to state and per-layer outputs. */
 int rr_ledger_views(rr_ledger* L, rr_views* out);
 
-/* Checkpoint / restore of the ledger (routes, sentinels, ages, kth_score, margin) to a host
- * blob of rr_export_bytes() bytes, laid out in that order, each array as in rr_views.
+/* Checkpoint / restore of the ledger -- the three row-major tensors of Section 4.1 (routes,
+ * sentinels, ages) plus the k-th score and margin recorded at each row's last routing -- to a
+ * host blob of rr_export_bytes() bytes, laid out in that order, each array as in rr_views.
  * Both synchronise `stream`. */
 int rr_export_bytes(const rr_config* cfg, size_t* bytes);
 int rr_ledger_export(rr_ledger* L, void* host_blob, size_t bytes, void* stream);

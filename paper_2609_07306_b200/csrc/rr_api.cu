@@ -177,6 +177,11 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
 
 void rr_count_launch(int n) { g_launches.fetch_add((unsigned long long)n); }
 
+std::mutex& rr_attr_mutex() {
+  static std::mutex mu;
+  return mu;
+}
+
 extern "C" {
 
 int rr_workspace_bytes(const rr_config* cfg, size_t* ledger_bytes, size_t* scratch_bytes) {
@@ -308,11 +313,13 @@ int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host
     for (auto e : evs)
       if (!*e) RR_CUDA(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
   }
-  // inputs of layer l -> staging set l%2 once layer l-2 has consumed it; issued one layer ahead
-  // so that the copy stream never queues an upload behind a download that waits for compute
+  // inputs of layer l -> staging set l%2 once its previous user has consumed it (layer l-2, or
+  // a layer of the previous call: the events live in the ledger, and waiting on an event that
+  // was never recorded returns at once); issued one layer ahead so that the copy stream never
+  // queues an upload behind a download that waits for compute
   auto upload = [&](int l) -> int {
     const int b = l & 1;
-    if (l >= 2) RR_CUDA(cudaStreamWaitEvent(cs, L->ev_consumed[b], 0));
+    RR_CUDA(cudaStreamWaitEvent(cs, L->ev_consumed[b], 0));
     RR_CUDA(cudaMemcpyAsync(dev_qc_staging[b], host_qc[l], qb, cudaMemcpyHostToDevice, cs));
     RR_CUDA(cudaMemcpyAsync(dev_kc_staging[b], host_kc[l], kb, cudaMemcpyHostToDevice, cs));
     RR_CUDA(cudaEventRecord(L->ev_copied[b], cs));
@@ -329,7 +336,7 @@ int rr_route_layers_host(rr_ledger* L, int32_t n_layers, const void* const* host
     if (l + 1 < n_layers) { rc = upload(l + 1); if (rc != RR_OK) return rc; }
     if (host_routes && host_routes[l]) {
       // snapshot on the compute stream (device to device), copy out on the download stream
-      if (l >= 2) RR_CUDA(cudaStreamWaitEvent(st, L->ev_d2h[b], 0));
+      RR_CUDA(cudaStreamWaitEvent(st, L->ev_d2h[b], 0));   // the staging set's last download
       RR_CUDA(cudaMemcpyAsync(dev_routes_staging[b], p.routes, rb, cudaMemcpyDeviceToDevice, st));
       RR_CUDA(cudaEventRecord(L->ev_snap[b], st));
       RR_CUDA(cudaStreamWaitEvent(ds, L->ev_snap[b], 0));

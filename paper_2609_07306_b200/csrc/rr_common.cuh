@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <mutex>
 #include <vector>
 #include "../../include/routerelay.h"
 
@@ -125,12 +126,18 @@ cudaError_t rr_launch_reset(const RRParams& p, cudaStream_t st);
 
 void rr_count_launch(int n = 1);
 
-// Function attributes (dynamic shared-memory limit) are per device: true the first time the
-// calling site runs on the current device.  `done` is the site's own bit mask of devices.
-inline bool rr_first_use_on_device(unsigned long long& done) {
+// Function attributes (dynamic shared-memory limit) are per device: `setup` runs the first time
+// the calling site is reached with a given device current, under a lock, and the device is
+// marked done only if it returned cudaSuccess (so a failure is retried, and no other host
+// thread launches before the attributes are in place).  `done` is the site's own bit mask.
+std::mutex& rr_attr_mutex();
+template <class F>
+inline cudaError_t rr_once_per_device(unsigned long long& done, F&& setup) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev > 63) return true;
-  if ((done >> dev) & 1ull) return false;
-  done |= 1ull << dev;
-  return true;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev > 63) return setup();
+  std::lock_guard<std::mutex> lock(rr_attr_mutex());
+  if ((done >> dev) & 1ull) return cudaSuccess;
+  const cudaError_t e = setup();
+  if (e == cudaSuccess) done |= 1ull << dev;
+  return e;
 }

@@ -320,16 +320,18 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
   e = rr_encode_tmap_bf16_3d(&tmap_q, qc, p.d, p.n_q, p.P, tcpipe::BM);
   if (e != cudaSuccess) return e;
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
-  if (rr_first_use_on_device(attr_done)) {
-    e = cudaFuncSetAttribute(rescore_dense_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = rr_once_per_device(attr_done, [] {
+    cudaError_t a = cudaFuncSetAttribute(rescore_dense_kernel<128>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (a != cudaSuccess) return a;
+    a = cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              227 * 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024);
-    if (e != cudaSuccess) return e;
+    if (a != cudaSuccess) return a;
     cudaFuncSetAttribute(rescore_dense_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  }
+    return cudaSuccess;
+  });
+  if (e != cudaSuccess) return e;
   const int grid = p.n_tiles;
   if (p.d == 128)
     rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words);

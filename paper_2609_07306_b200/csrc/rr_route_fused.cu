@@ -1114,14 +1114,16 @@ cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void*
   const int keep = p.k + (p.m > 0 ? p.m : 1);
   const bool fine = cap - keep < 64;             // little room above keep: check the fill more often
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
-  if (rr_first_use_on_device(attr_done)) {
+  e = rr_once_per_device(attr_done, [] {
     const void* fns[4] = {(const void*)route_fused_kernel<128, 32>, (const void*)route_fused_kernel<128, 8>,
                           (const void*)route_fused_kernel<64, 32>, (const void*)route_fused_kernel<64, 8>};
     for (const void* fn : fns) {
-      e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
+      const cudaError_t a = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (a != cudaSuccess) return a;
     }
-  }
+    return cudaSuccess;
+  });
+  if (e != cudaSuccess) return e;
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   if (p.d == 128 && !fine)
     route_fused_kernel<128, 32><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, cap, aux);

@@ -227,14 +227,15 @@ cudaError_t rr_launch_score_tc(const RRParams& p, const void* qc, const void* kc
   if (e != cudaSuccess) return e;
   const int grid = p.P * p.tiles_per_problem;
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
-  if (rr_first_use_on_device(attr_done)) {
-    e = cudaFuncSetAttribute(score_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg<128>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg<64>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-  }
+  e = rr_once_per_device(attr_done, [] {
+    const cudaError_t a = cudaFuncSetAttribute(score_tc_kernel<128>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               Cfg<128>::SMEM_BYTES);
+    if (a != cudaSuccess) return a;
+    return cudaFuncSetAttribute(score_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Cfg<64>::SMEM_BYTES);
+  });
+  if (e != cudaSuccess) return e;
   if (p.d == 128)
     score_tc_kernel<128><<<grid, NT, Cfg<128>::SMEM_BYTES, st>>>(p, (const __nv_bfloat16*)qc, tmap,
                                                                   row_list);

@@ -194,11 +194,11 @@ cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int 
   const int nk_pad = (p.n_k + 31) & ~31;
   const size_t smem = (size_t)WARPS * (nk_pad + 256 + nk_pad / 32) * sizeof(uint32_t);
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
-  if (rr_first_use_on_device(attr_done)) {
-    cudaError_t e = cudaFuncSetAttribute(topk_rows_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    if (e != cudaSuccess) return e;
-  }
+  const cudaError_t e = rr_once_per_device(attr_done, [] {
+    return cudaFuncSetAttribute(topk_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                96 * 1024);
+  });
+  if (e != cudaSuccess) return e;
   const int grid = (p.rows + WARPS - 1) / WARPS;
   topk_rows_kernel<<<grid, WARPS * 32, smem, st>>>(p, row_list, (uint32_t)layer);
   rr_count_launch();

@@ -15,6 +15,8 @@ the outputs are compared:
   identical whenever route and near-miss sets are; margin within tolerance
 * rows stable on both sides: route and sentinel rows bit-identical to the previous layer,
   age advanced by one
+* with token expansion on: the token ranges of every checked row equal the oracle's expansion
+  of the DEVICE's routes (Section 2.1), bit for bit, every layer
 """
 from __future__ import annotations
 
@@ -54,6 +56,7 @@ class ParityReport:
     flag_mismatch_ambiguous: int = 0
     route_mismatch_ambiguous: int = 0
     hard_mismatches: int = 0
+    token_range_rows: int = 0
     max_score_err: float = 0.0
     max_score_rel_err: float = 0.0
     notes: List[str] = dataclasses.field(default_factory=list)
@@ -105,6 +108,9 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
             led.sentinels[sel_t] = torch.from_numpy(oracle_led.sentinels).cuda()
             led.ages[sel_t] = torch.from_numpy(oracle_led.ages).cuda()
             led.margin[sel_t] = torch.from_numpy(oracle_led.margin.astype(np.float32)).cuda()
+            if w.chunk_tokens > 0:      # the ranges belong to the routes that were just imported
+                led.token_ranges[sel_t] = torch.from_numpy(O.token_ranges(
+                    oracle_led.routes, w.chunk_tokens, coalesce=bool(w.coalesce_ranges))).cuda()
             prev_gpu_routes = led.routes.clone()
             prev_gpu_sent = led.sentinels.clone()
             prev_gpu_ages = led.ages.clone()
@@ -222,9 +228,29 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
             if np.isfinite(om) != np.isfinite(g_margin[ri]) or \
                     (np.isfinite(om) and abs(g_margin[ri] - om) > amb_tol[ri]):
                 rep.bad(f"layer {l} row {ri}: margin differs ({g_margin[ri]} vs {om})")
+        if w.chunk_tokens > 0:
+            # stable rows keep the ranges of the layer that routed them, so every checked row
+            # must carry the expansion of its current route
+            g_ranges = _gpu_rows(led.token_ranges, rows_sel)
+            want = O.token_ranges(g_routes, w.chunk_tokens, coalesce=bool(w.coalesce_ranges))
+            rep.token_range_rows += len(rows_sel)
+            if not np.array_equal(g_ranges, want):
+                badrows = np.nonzero((g_ranges != want).any(axis=(1, 2)))[0]
+                rep.bad(f"layer {l}: token ranges differ from the expansion of the device's "
+                        f"routes on {len(badrows)} rows (first: {badrows[:4].tolist()})")
         oracle_led = res.ledger
     led.close()
     return rep
+
+
+def summary_line(rep: ParityReport) -> str:
+    """One line with the counts the parity protocol asks to be reported."""
+    return (f"rows {rep.rows_checked} refreshed {rep.refreshed_checked} | ambiguous flag rows "
+            f"{rep.ambiguous_flag_rows} (mismatching {rep.flag_mismatch_ambiguous}) | ambiguous "
+            f"route rows {rep.ambiguous_route_rows} (mismatching {rep.route_mismatch_ambiguous}) | "
+            f"ambiguous near-miss rows {rep.ambiguous_near_rows} | token-range rows "
+            f"{rep.token_range_rows} | max |score err| {rep.max_score_err:.3e} "
+            f"rel {rep.max_score_rel_err:.3e}")
 
 
 def assert_clean(rep: ParityReport, max_ambiguous_fraction: float = 0.02):

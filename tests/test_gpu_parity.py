@@ -12,11 +12,13 @@ from paper_2609_07306_b200.ledger import RouteLedger, config_from_workload, devi
 pytestmark = pytest.mark.gpu
 
 
-def _report(rep):
-    print(f"rows {rep.rows_checked} refreshed {rep.refreshed_checked} | ambiguous flag rows "
-          f"{rep.ambiguous_flag_rows} (mismatching {rep.flag_mismatch_ambiguous}) | ambiguous "
-          f"route rows {rep.ambiguous_route_rows} (mismatching {rep.route_mismatch_ambiguous}) | "
-          f"max |score err| {rep.max_score_err:.3e} rel {rep.max_score_rel_err:.3e}")
+def _report(rep, record_property=None, name="parity"):
+    """Prints the counts of ambiguous / soft-mismatching rows and, when the test passes pytest's
+    record_property fixture, stores them with the test's result (junit / report plugins)."""
+    line = parity.summary_line(rep)
+    print(line)
+    if record_property is not None:
+        record_property(name, line)
 
 
 def test_tiny_fp32_all_layers():
@@ -65,26 +67,37 @@ def test_long_context_shape_small():
         rep = parity.run_teacher_forced(w, two_pass=two_pass, gathered=gathered)
         _report(rep)
         parity.assert_clean(rep)
+        assert rep.token_range_rows == 3 * w.rows
+    # the same with runs of adjacent chunks merged (k = 64: the multi-block coalescing path)
+    rep = parity.run_teacher_forced(w.replace(coalesce_ranges=True))
+    _report(rep)
+    parity.assert_clean(rep)
+    assert rep.token_range_rows == 3 * w.rows
 
 
-def test_high_drift_full_size_sampled_problems():
-    """BASELINE configuration 4 at full size (256 problems x 1024 rows, the launch the
-    benchmark times), first 5 layers (anchor, 3 relays, relay after a centroid re-draw);
-    three problems are checked row by row against the oracle, the integer work (compaction,
-    ages, stable rows) on all 262144 rows."""
+def test_high_drift_full_size_sampled_problems(record_property):
+    """The high-drift configuration at full size (batch 8 x 32 heads = 256 problems of 1024 x
+    1024 chunks, k/m/r = 32/16/16: the launch the benchmark times), layers 0-9: the first
+    anchor, relays before and after the centroid re-draws at layers 4 and 8, the second anchor
+    at layer 8 and the relay after it.  Eight problems are checked row by row against the oracle,
+    the integer work (compaction, ages, stable rows) on all 262144 rows."""
     w = W.high_drift()
-    rep = parity.run_teacher_forced(w, check_problems=[0, 101, 255], layers=5, gen_threads=16)
-    _report(rep)
+    rep = parity.run_teacher_forced(w, check_problems=[0, 37, 74, 101, 128, 190, 233, 255],
+                                    layers=10, gen_threads=16)
+    _report(rep, record_property, "high_drift_full_size")
     parity.assert_clean(rep)
 
 
-def test_long_context_full_size_sampled_problems():
-    """BASELINE configuration 5 at full size (64 problems x 2048 rows), 3 layers, two
-    problems checked against the oracle."""
+def test_long_context_full_size_sampled_problems(record_property):
+    """The long-context configuration at full size (64 problems x 2048 chunks, k/m/r =
+    64/32/32, 64-token chunks expanded to token ranges), 3 layers, eight problems checked
+    against the oracle, token ranges included."""
     w = W.long_ctx()
-    rep = parity.run_teacher_forced(w, check_problems=[3, 60], layers=3, gen_threads=16)
-    _report(rep)
+    rep = parity.run_teacher_forced(w, check_problems=[0, 3, 17, 26, 35, 44, 53, 63], layers=3,
+                                    gen_threads=16)
+    _report(rep, record_property, "long_ctx_full_size")
     parity.assert_clean(rep)
+    assert rep.token_range_rows == 3 * 8 * w.n_q
 
 
 def test_degenerate_all_equal_scores():
@@ -194,6 +207,40 @@ def test_pipelined_host_layers_entry_point():
     led.close(); ref.close()
 
 
+def test_pipelined_host_layers_back_to_back_calls():
+    """Two rr_route_layers_host calls on the same ledger and staging buffers with NO
+    synchronisation between them (what a serving loop does): the second call's uploads must
+    wait for the first call's last readers of each staging set.  The first call routes other
+    inputs, so a staging set overwritten too early (or too late) shows in the routes."""
+    w = W.sweep(512, 0.15).replace(heads=8, layers=5, anchor_every=3)
+    L = w.layers
+    q, k = W.generate(w)
+    q2, k2 = W.generate(w.replace(seed=9))
+    led = RouteLedger(config_from_workload(w))
+    ref = RouteLedger(config_from_workload(w))
+    pin = lambda x: torch.from_numpy(x.view(np.int16)).pin_memory()
+    hq, hk = [pin(q[l]) for l in range(L)], [pin(k[l]) for l in range(L)]
+    hq2, hk2 = [pin(q2[l]) for l in range(L)], [pin(k2[l]) for l in range(L)]
+    dq = [torch.empty_like(hq[0], device="cuda") for _ in range(2)]
+    dk = [torch.empty_like(hk[0], device="cuda") for _ in range(2)]
+    dr = [torch.empty(w.rows, w.k, dtype=torch.int32, device="cuda") for _ in range(2)]
+    outs1 = [torch.empty(w.rows, w.k, dtype=torch.int32).pin_memory() for _ in range(L)]
+    outs2 = [torch.empty(w.rows, w.k, dtype=torch.int32).pin_memory() for _ in range(L)]
+    cs, ds = torch.cuda.Stream(), torch.cuda.Stream()
+    anchors = [w.is_anchor(l) for l in range(L)]
+    for rep_ in range(3):                        # a few rounds: a race need not show at once
+        led.reset()
+        led.route_layers_host(hq2, hk2, anchors, 0, dq, dk, dr, outs1, cs, ds)
+        led.route_layers_host(hq, hk, anchors, 0, dq, dk, dr, outs2, cs, ds)   # no sync before
+        torch.cuda.synchronize()
+        ref.reset()
+        for l in range(L):
+            (ref.route_anchor if anchors[l] else ref.route_relay)(device_tensor(q[l]), device_tensor(k[l]), l)
+            torch.cuda.synchronize()
+            assert torch.equal(outs2[l], ref.routes.cpu()), f"round {rep_} layer {l}"
+    led.close(); ref.close()
+
+
 @pytest.mark.parametrize("coalesce", [False, True], ids=["per_chunk", "coalesced"])
 @pytest.mark.parametrize("two_pass", [False, True], ids=["fused", "two_pass"])
 def test_token_ranges(two_pass, coalesce):
@@ -214,10 +261,12 @@ def test_token_ranges(two_pass, coalesce):
     led.close()
 
 
-def test_free_running_summary_matches_oracle():
+@pytest.mark.parametrize("wl", ["moderate", "sweep_1024_rho0.30_4heads"])
+def test_free_running_summary_matches_oracle(wl):
     """All layers without teacher forcing: recall / refreshed-row / score-pair fractions of
-    the device run agree with the oracle's run up to the ambiguous rows."""
-    w = W.moderate()
+    the device run agree with the oracle's run up to the ambiguous rows.  Second case: the
+    routing-scale sweep at 1024 chunks and the highest drift (4 of its 32 heads, 16 layers)."""
+    w = W.moderate() if wl == "moderate" else W.sweep(1024, 0.30).replace(heads=4)
     q, k = W.generate(w)
     p = parity.oracle_params(w)
     res, summ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),

@@ -451,3 +451,77 @@ def test_minimum_reuse_horizon_invariant():
         assert not both.any()
         seen += int(res[l].flags.sum())
     assert seen > 0
+
+
+# ------------------------------------------------------------------ recall and run-level accounting
+def test_recall_counts_partial_overlap_hand_case():
+    """Section 5: recall compares the reused chunk ids with the exact per-layer top-k.
+    Hand-worked rows with partial overlap, -1 padding on either side and different valid widths."""
+    routes = np.array([[3, 5, -1], [0, 1, 2], [4, -1, -1], [7, 8, 9]], np.int32)
+    full = np.array([[5, 7, -1], [2, 1, 0], [4, -1, -1], [1, 2, -1]], np.int32)
+    # row 0: {3,5} vs {5,7} -> 1 of 2; row 1: 3 of 3; row 2: 1 of 1; row 3: {7,8,9} vs {1,2} -> 0 of 2
+    assert O.recall_counts(routes, full) == (5, 8)
+    # the denominator is the size of the exact set, not of the reused one
+    assert O.recall_counts(np.array([[1, 2, 3]], np.int32), np.array([[3, -1, -1]], np.int32)) == (1, 1)
+    assert O.recall_counts(np.array([[3, -1, -1]], np.int32), np.array([[1, 2, 3]], np.int32)) == (1, 3)
+    # a -1 on both sides is padding, never a hit
+    assert O.recall_counts(np.array([[-1, -1]], np.int32), np.array([[-1, -1]], np.int32)) == (0, 0)
+
+
+def test_run_recall_hand_worked():
+    """Whole run whose recall is known by hand: d = 1, 4 key chunks, k = 2, no sentinels (so the
+    relay layer can only reuse), one anchor.  Keys (4,3,2,1) then (4,2,3,1); query rows +1, 0, -1.
+    Layer 0 routes {0,1}, {0,1} (all ties -> smallest ids), {3,2}; exact top-2 at layer 1:
+    {0,2}, {0,1}, {3,1} -> hits 1 + 2 + 1 of 6 on the relay layer, 10 of 12 over the run."""
+    p = O.OracleParams(n_q=3, n_k=4, k=2, m=0, r=0)
+    q = np.array([[[1.0], [0.0], [-1.0]]])
+    k0 = np.array([[[4.0], [3.0], [2.0], [1.0]]])
+    k1 = np.array([[[4.0], [2.0], [3.0], [1.0]]])
+    res, summ = O.run_layers(np.stack([q, q]), np.stack([k0, k1]), p, anchor_every=8)
+    assert [sorted(r) for r in res[0].ledger.routes.tolist()] == [[0, 1], [0, 1], [2, 3]]
+    assert [sorted(r) for r in res[1].full_routes.tolist()] == [[0, 2], [0, 1], [1, 3]]
+    assert not res[1].flags.any()                       # nothing can challenge a route
+    assert summ.recall_relay == pytest.approx(4 / 6, abs=1e-15)
+    assert summ.recall_all == pytest.approx(10 / 12, abs=1e-15)
+    assert summ.rerouted_fraction == pytest.approx(0.5) and summ.flagged_relay_fraction == 0.0
+    # score pairs: anchor 3 rows x 4, relay 3 rows x 2 candidates, over 2 x 12
+    assert summ.score_pair_fraction == pytest.approx((12 + 6) / 24)
+
+
+@pytest.mark.parametrize("L,n_k,k", [(4, 32, 3), (6, 64, 12), (3, 16, 16)])
+def test_run_accounting_fixed_stride_closed_form(L, n_k, k):
+    """Run-level score pairs of the ORACLE's own run with m = r = 0 and a single anchor, no
+    mask: 1/L + (L-1)/L * k/n_k (the arithmetic of the sentinel-ablation table, Section 5.2)."""
+    rng = np.random.default_rng(L * 1000 + n_k)
+    q = rng.standard_normal((L, 2, 9, 8))
+    kk = rng.standard_normal((L, 2, n_k, 8))
+    p = O.OracleParams(n_q=9, n_k=n_k, k=k, m=0, r=0)
+    res, summ = O.run_layers(q, kk, p, anchor_every=10 ** 6)
+    assert summ.score_pair_fraction == pytest.approx(1 / L + (L - 1) / L * k / n_k, abs=1e-15)
+    assert summ.rerouted_fraction == pytest.approx(1 / L, abs=1e-15)
+    c = summ.counters
+    assert c["cand_pairs"] == (L - 1) * 2 * 9 * k and c["full_pairs"] == 2 * 9 * n_k
+    assert c["anchor_rows"] == 18 and c["relay_rows"] == (L - 1) * 18 and c["flagged_rows"] == 0
+
+
+def test_run_accounting_causal_candidate_pairs():
+    """Under the causal mask every relay layer charges every row min(v_i, c) candidate pairs
+    (route, near-miss and random slots that exist), every flagged row v_i more; anchors charge
+    v_i per row.  Asserted on the oracle's run-level counters against the flags it reports."""
+    w = W.moderate().replace(heads=2, layers=5, anchor_every=3)
+    p, res, summ = _run(w, [0, 1])
+    v = np.tile(p.valid_counts(), 2)
+    c = summ.counters
+    n_relay = sum(not r.is_anchor for r in res)
+    n_anchor = len(res) - n_relay
+    assert n_relay == 3 and n_anchor == 2
+    assert c["cand_pairs"] == n_relay * int(np.minimum(v, p.c).sum())
+    flagged_v = sum(int(v[r.flags != 0].sum()) for r in res if not r.is_anchor)
+    assert flagged_v > 0
+    assert c["full_pairs"] == n_anchor * int(v.sum()) + flagged_v
+    assert c["dense_pairs"] == len(res) * int(v.sum())
+    assert summ.score_pair_fraction == pytest.approx(
+        (c["cand_pairs"] + c["full_pairs"]) / (len(res) * v.sum()), abs=1e-15)
+    # the per-row candidate count the run used equals the closed form slot by slot
+    led = res[0].ledger
+    assert np.array_equal(O.valid_candidate_counts(led), np.minimum(v, p.c))

@@ -45,6 +45,31 @@ def test_noalloc_compaction_matches_relay_twice_in_a_row():
     led.close()
 
 
+def test_noalloc_ragged_tiles_against_nonzero():
+    """Problems whose row count is not a multiple of the 128-row tile (200 rows, 3 problems: a
+    full tile and a ragged one per problem), twice in a row with different flag patterns:
+    list, count and per-problem offsets against numpy.nonzero of the flags."""
+    n_problems, n_q = 3, 200
+    rng = np.random.default_rng(5)
+    rows_out = torch.empty(n_problems * n_q, dtype=torch.int32, device="cuda")
+    count_out = torch.empty(1, dtype=torch.int32, device="cuda")
+    offs_out = torch.empty(n_problems + 1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    for density in (0.3, 0.9):
+        flags = (rng.random(n_problems * n_q) < density).astype(np.uint8) * 3   # any non-zero counts
+        dflags = torch.from_numpy(flags).cuda()
+        rows_out.fill_(-7)
+        B.rr_compact_flags_noalloc(dflags.data_ptr(), n_problems, n_q, rows_out.data_ptr(),
+                                   count_out.data_ptr(), offs_out.data_ptr(), stream)
+        torch.cuda.synchronize()
+        nz = np.nonzero(flags)[0]
+        assert int(count_out.item()) == len(nz)
+        assert np.array_equal(rows_out[:len(nz)].cpu().numpy(), nz)
+        assert (rows_out[len(nz):] == -7).all()
+        per_problem = (flags != 0).reshape(n_problems, n_q).sum(axis=1)
+        assert np.array_equal(offs_out.cpu().numpy(), np.concatenate([[0], np.cumsum(per_problem)]))
+
+
 def test_noalloc_rejects_oversize_and_bad_arguments():
     flags = torch.zeros(256, dtype=torch.uint8, device="cuda")
     out = torch.zeros(256, dtype=torch.int32, device="cuda")
