@@ -79,7 +79,11 @@ typedef struct rr_config {
                               bit 1: route through the two-pass path (score rows in scratch
                               + warp-level TopK) even where the fused kernel applies;
                               bit 2: rescore candidates with the gathered FP32 kernel even
-                              where the tensor-core strip kernel applies                  */
+                              where the tensor-core strip kernel applies;
+                              bit 3 (tests): the two-sweep routing kernel hands every fifth
+                              row to its exact slow path;
+                              bit 4: route with the streaming fused kernel even where the
+                              two-sweep kernel applies                                     */
   /* Optional policies either side of the trigger; all zero = the plain method.             */
   int32_t global_sentinels;/* mandatory global candidates (Section 3.1, item 3): bit 0 = the
                               sink chunk 0, bit 1 = the most recent chunk the row may select.

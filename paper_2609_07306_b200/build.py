@@ -36,20 +36,34 @@ def is_stale() -> bool:
 
 
 def build(verbose: bool = False, force: bool = False) -> str:
+    """One nvcc process per source file (in parallel) into a scratch folder, then one link."""
     if not force and not is_stale():
         return LIB
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
-           "-std=c++17", "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-           "-o", LIB] + os.environ.get("RR_EXTRA_NVCC_FLAGS", "").split() + sources()
+    import tempfile
+    from concurrent.futures import ThreadPoolExecutor
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC"] + os.environ.get("RR_EXTRA_NVCC_FLAGS", "").split()
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-        print(" ".join(cmd))
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        flags += ["-Xptxas", "-v"]
+    nvcc = _nvcc()
+    with tempfile.TemporaryDirectory(prefix="rr_build_") as tmp:
+        def compile_one(src):
+            obj = os.path.join(tmp, os.path.basename(src)[:-3] + ".o")
+            res = subprocess.run([nvcc] + flags + ["-c", src, "-o", obj], capture_output=True,
+                                 text=True)
+            return src, obj, res
+        with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+            done = list(ex.map(compile_one, sources()))
+        log = "".join(f"== {os.path.basename(s)}\n{r.stdout}{r.stderr}" for s, _, r in done)
+        if any(r.returncode != 0 for _, _, r in done):
+            raise RuntimeError("nvcc failed:\n" + log)
+        res = subprocess.run([nvcc, "-shared", "-cudart", "static", "-gencode",
+                              "arch=compute_100a,code=sm_100a", "-o", LIB] + [o for _, o, _ in done],
+                             capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     if verbose:
-        print(res.stdout + res.stderr)
+        print(log)
     return LIB
 
 

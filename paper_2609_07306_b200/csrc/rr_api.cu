@@ -79,8 +79,12 @@ RRParams shape_params(const rr_config* cfg) {
   return p;
 }
 
+bool uses_sweep(const rr_config* cfg) {
+  return !(cfg->debug_outputs & (2 | 16)) && rr_route_sweep_supported(shape_params(cfg));
+}
+
 bool uses_fused(const rr_config* cfg) {
-  return !(cfg->debug_outputs & 2) && rr_route_fused_supported(shape_params(cfg));
+  return !(cfg->debug_outputs & 2) && !uses_sweep(cfg) && rr_route_fused_supported(shape_params(cfg));
 }
 
 Layout make_layout(const rr_config* c) {
@@ -111,7 +115,7 @@ Layout make_layout(const rr_config* c) {
   L.token_ranges = o;    o = align_up(o + (c->chunk_tokens > 0 ? rows * c->k * 8 : 0));
   L.cand_scores = o;     o = align_up(o + ((c->debug_outputs & 1) ? rows * cw * 4 : 0));
   // score rows are only materialised by the two-pass path
-  L.S = o;               o = align_up(o + (uses_fused(c) ? 0 : rows * (size_t)c->n_k * 4));
+  L.S = o;               o = align_up(o + (uses_fused(c) || uses_sweep(c) ? 0 : rows * (size_t)c->n_k * 4));
   L.scratch_total = o;
   return L;
 }
@@ -144,7 +148,10 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
   if (anchor) {
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
     LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, L->dense_pairs_per_layer, st));
-    if (L->fused) {
+    if (L->sweep) {
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer,
+                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+    } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, nullptr, layer, st));
     } else {
       if (p.dtype == RR_BF16) LAUNCH(RR_KIND_SCORE_TC, rr_launch_score_tc(p, qc, kc, nullptr, st));
@@ -158,7 +165,10 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     if (L->dense_rescore) LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, st));
     else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
-    if (L->fused) {
+    if (L->sweep) {
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, p.refresh_rows, layer,
+                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+    } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
     } else {
       if (p.dtype == RR_BF16)
@@ -238,6 +248,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.token_ranges = cfg->chunk_tokens > 0 ? (int32_t*)(sb + lay.token_ranges) : nullptr;
   p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
+  L->sweep = uses_sweep(cfg);
   L->fused = uses_fused(cfg);
   L->dense_rescore = !(cfg->debug_outputs & 4) && rr_rescore_dense_supported(p);
   *out = L;

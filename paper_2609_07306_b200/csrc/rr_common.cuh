@@ -39,7 +39,8 @@ struct rr_ledger {
   size_t export_bytes;
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
-  bool fused;                              // full routing runs in the fused tensor-core kernel
+  bool sweep;                              // full routing runs in the two-sweep fused kernel
+  bool fused;                              // ... else in the streaming fused kernel
   bool dense_rescore;                      // relay rescoring reads the tensor-core score strip
   unsigned long long dense_pairs_per_layer;
   // benchmark-only per-kernel timing
@@ -110,6 +111,10 @@ cudaError_t rr_launch_score_tc(const RRParams& p, const void* qc, const void* kc
 bool rr_route_fused_supported(const RRParams& p);
 cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void* kc,
                                   const int32_t* row_list, int layer, cudaStream_t st);
+bool rr_route_sweep_supported(const RRParams& p);
+cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void* kc,
+                                  const int32_t* row_list, int layer, int force_hard,
+                                  cudaStream_t st);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
 cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,

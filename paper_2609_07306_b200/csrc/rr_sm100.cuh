@@ -53,6 +53,40 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   *abort_flag = 1u;
   return false;
 }
+// Bounded wait without sleeping, for the single threads whose hand-offs are on the critical
+// path of a tile pipeline (TMA producer, MMA issuer): a sleep quantum between polls would be
+// added to every tile.  The limit is counted in polls (a failed try_wait itself blocks for a
+// hardware-defined slice, so this is of the order of a second).
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity,
+                                               volatile uint32_t* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && *abort_flag) return false;
+  }
+  *abort_flag = 1u;
+  return false;
+}
+// For waits that usually last hundreds of cycles and are made by many warps at once (the
+// consumers of a tile pipeline whose per-tile work is short): one lane polls, sleeping between
+// polls, and the warp follows it -- 32 lanes polling in a tight loop from 16 warps keep the
+// shared-memory port and the issue slots busy that the producer side needs.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity,
+                                               volatile uint32_t* abort_flag, uint32_t ns) {
+  bool ok = false;
+  if ((threadIdx.x & 31) == 0) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+      if (mbar_try_wait(bar, parity)) { ok = true; break; }
+      if (*abort_flag) break;
+      __nanosleep(ns);
+    }
+    if (!ok && !*abort_flag) *abort_flag = 1u;
+  }
+  ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+  // the other lanes have not observed the phase themselves: one (successful) test each
+  // orders their later reads behind the barrier's completion
+  if (ok && (threadIdx.x & 31) != 0) ok = mbar_try_wait(bar, parity);
+  return ok;
+}
 // The same for the roles that run far ahead of the consumers (the TMA producer and the MMA
 // issuer): they sleep between polls from the first miss on, so that their polling does not take
 // issue slots from the warps that share their schedulers.
@@ -87,6 +121,13 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* t
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z),
         "r"(smem_u32(bar))
       : "memory");
+}
+// The same tile fetched into L2 only (no shared-memory destination, no barrier): hides the
+// DRAM latency of a tile that a later tma_load_3d will ask for.
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* tmap, int x, int y, int z) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z)
+               : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");

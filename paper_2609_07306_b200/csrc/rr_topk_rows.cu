@@ -7,60 +7,11 @@
 // resolved towards the smaller chunk id by walking the row in index order with ballots.
 // Input: score rows S[slot, 0..v) in global memory (fp32), slot = position in the refresh
 // list (relay) or the global row id (anchor).
-#include "rr_common.cuh"
+#include "rr_warp_topk.cuh"
 
 namespace {
 
 constexpr int WARPS = 4;
-constexpr unsigned FULL = 0xFFFFFFFFu;
-
-struct Sel { uint32_t key; int need; int ties; };
-
-// Key of rank T (1-based, descending) among keys[0..v): `need` of the `ties` keys equal to
-// it belong to the top T.  Requires 1 <= T <= v.
-__device__ Sel warp_select(const uint32_t* keys, int v, int T, uint32_t* hist, int lane) {
-  uint32_t prefix = 0, mask = 0;
-  int need = T, ties = 0;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = lane; b < 256; b += 32) hist[b] = 0;
-    __syncwarp();
-    for (int j = lane; j < v; j += 32) {
-      uint32_t key = keys[j];
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-    }
-    __syncwarp();
-    // lane owns digits 255-8*lane .. 248-8*lane, walked in descending order
-    int loc[8], sum = 0;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) { loc[q] = (int)hist[255 - 8 * lane - q]; sum += loc[q]; }
-    int incl = sum;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      int t = __shfl_up_sync(FULL, incl, off);
-      if (lane >= off) incl += t;
-    }
-    int excl = incl - sum;
-    bool mine = (excl < need) && (need <= incl);
-    int dsel = 0, before = 0, cnt = 0, run = excl;
-    bool found = false;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      bool here = mine && !found && (need <= run + loc[q]);
-      if (here) { dsel = 255 - 8 * lane - q; before = run; cnt = loc[q]; found = true; }
-      run += loc[q];
-    }
-    int src = __ffs(__ballot_sync(FULL, mine)) - 1;
-    dsel = __shfl_sync(FULL, dsel, src);
-    before = __shfl_sync(FULL, before, src);
-    cnt = __shfl_sync(FULL, cnt, src);
-    need -= before;
-    prefix |= (uint32_t)dsel << shift;
-    mask |= 0xFFu << shift;
-    ties = cnt;
-    __syncwarp();
-  }
-  return Sel{prefix, need, ties};
-}
 
 __global__ void __launch_bounds__(WARPS * 32)
 topk_rows_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t layer) {
@@ -79,112 +30,9 @@ topk_rows_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t laye
   const int i = g % p.n_q;
   const int v = rr_valid_count(i, p.n_k, p.causal, p.causal_offset);
   const float* srow = p.S + (size_t)slot * p.n_k;
-  const unsigned lt = (1u << lane) - 1u;
-
   for (int j = lane; j < v; j += 32) keys[j] = rr_order_key(srow[j]);
-  for (int w = lane; w < nk_pad / 32; w += 32) bitmap[w] = 0;
   __syncwarp();
-
-  const int Tk = min(p.k, v), Tkeep = min(p.k + p.m, v);
-  const Sel sk = warp_select(keys, v, Tk, hist, lane);
-  const Sel sn = (Tkeep > Tk) ? warp_select(keys, v, Tkeep, hist, lane) : sk;
-
-  int32_t* route = p.routes + (size_t)g * p.k;
-  int32_t* sent = p.sentinels + (size_t)g * p.sw;
-  int run_eqk = 0, run_eqn = 0, run_route = 0, run_near = 0;
-  for (int j0 = 0; j0 < v; j0 += 32) {
-    const int j = j0 + lane;
-    const bool valid = j < v;
-    const uint32_t key = valid ? keys[j] : 0u;
-    const bool eqk = valid && key == sk.key;
-    const bool eqn = valid && key == sn.key;
-    const unsigned bk = __ballot_sync(FULL, eqk), bn = __ballot_sync(FULL, eqn);
-    const int rank_k = run_eqk + __popc(bk & lt), rank_n = run_eqn + __popc(bn & lt);
-    const bool in_route = valid && (key > sk.key || (eqk && rank_k < sk.need));
-    const bool in_near = valid && !in_route && Tkeep > Tk &&
-                         (key > sn.key || (eqn && rank_n < sn.need));
-    const unsigned br = __ballot_sync(FULL, in_route), bnr = __ballot_sync(FULL, in_near);
-    if (in_route) route[run_route + __popc(br & lt)] = j;
-    if (in_near) sent[run_near + __popc(bnr & lt)] = j;
-    if (lane == 0) bitmap[j0 >> 5] = br | bnr;
-    run_eqk += __popc(bk); run_eqn += __popc(bn);
-    run_route += __popc(br); run_near += __popc(bnr);
-  }
-  for (int s = run_route + lane; s < p.k; s += 32) route[s] = -1;
-  for (int s = run_near + lane; s < p.m; s += 32) sent[s] = -1;
-
-  // k-th score and margin (min selected - max unselected)
-  float kth = rr_key_to_float(sk.key), margin = __int_as_float(0x7f800000);
-  if (v > Tk) {
-    uint32_t next = sk.key;
-    if (sk.ties <= sk.need) {
-      uint32_t best = 0;
-      for (int j = lane; j < v; j += 32) {
-        uint32_t key = keys[j];
-        if (key < sk.key && key > best) best = key;
-      }
-#pragma unroll
-      for (int off = 16; off; off >>= 1) best = max(best, __shfl_xor_sync(FULL, best, off));
-      next = best;
-    }
-    margin = kth - rr_key_to_float(next);
-  }
-  if (lane == 0) { p.kth[g] = kth; p.margin[g] = margin; }
-  __syncwarp();
-
-  // random sentinels: r distinct chunks from the valid ones outside route and near-miss
-  // mandatory global sentinels (sink chunk, most recent chunk): a slot each after the random
-  // ones, empty if the chunk is already in the route or a near-miss sentinel
-  int pool = v - Tkeep;
-  if (p.n_global) {
-    int gi = 0;
-    for (int b = 0; b < 2; ++b) {
-      if (!((p.global_mask >> b) & 1)) continue;
-      const int j = b == 0 ? 0 : v - 1;
-      int id = -1;
-      if (v > 0) {
-        const uint32_t word = bitmap[j >> 5], bit = 1u << (j & 31);
-        if (!(word & bit)) { id = j; --pool; }
-        __syncwarp();
-        if (id >= 0 && lane == 0) bitmap[j >> 5] = word | bit;
-        __syncwarp();
-      }
-      if (lane == 0) sent[p.m + p.r + gi] = id;
-      ++gi;
-    }
-  }
-  int32_t* rnd = sent + p.m;
-  int taken = 0;
-  if (p.r > 0 && pool > 0) {
-    if (pool > p.r) {
-      const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
-      const int limit = 64 * p.r;
-      for (int t0 = 0; t0 < limit && taken < p.r; t0 += 32) {
-        const uint32_t u = rr_draw_u32(rk, layer, (uint32_t)(t0 + lane));
-        const int jmine = (int)__umulhi(u, (uint32_t)v);
-        for (int l = 0; l < 32 && taken < p.r && t0 + l < limit; ++l) {
-          const int jj = __shfl_sync(FULL, jmine, l);
-          const uint32_t word = bitmap[jj >> 5];
-          const uint32_t bit = 1u << (jj & 31);
-          if (!(word & bit)) {
-            if (lane == 0) { bitmap[jj >> 5] = word | bit; rnd[taken] = jj; }
-            ++taken;
-          }
-          __syncwarp();
-        }
-      }
-    }
-    // whole pool (pool <= r) or the bounded-work fill: smallest free chunks first
-    for (int j0 = 0; j0 < v && taken < p.r; j0 += 32) {
-      const int j = j0 + lane;
-      const bool fr = j < v && !((bitmap[j0 >> 5] >> lane) & 1u);
-      const unsigned bf = __ballot_sync(FULL, fr);
-      const int pos = taken + __popc(bf & lt);
-      if (fr && pos < p.r) rnd[pos] = j;
-      taken = min(p.r, taken + __popc(bf));
-    }
-  }
-  for (int s = taken + lane; s < p.r; s += 32) rnd[s] = -1;
+  warptopk::route_row(p, keys, hist, bitmap, g, v, layer, lane);
 }
 
 }  // namespace

@@ -45,6 +45,51 @@ def test_sweep_shapes(n, two_pass, gathered):
     parity.assert_clean(rep)
 
 
+@pytest.mark.parametrize("variant", ["slow_rows", "streaming"])
+@pytest.mark.parametrize("wl", ["moderate", "sweep512", "sweep1024"])
+def test_routing_kernel_variants(wl, variant):
+    """The two other ways a bf16 row can be routed in one kernel: the two-sweep kernel with every
+    fifth row handed to its exact slow path (complete score row in shared memory + warp-level
+    radix select), and the streaming kernel that serves the shapes the two-sweep kernel does
+    not hold."""
+    w = {"moderate": W.moderate(),
+         "sweep512": W.sweep(512, 0.15).replace(heads=4, layers=4, anchor_every=3),
+         "sweep1024": W.sweep(1024, 0.30).replace(heads=3, layers=3, anchor_every=2)}[wl]
+    rep = parity.run_teacher_forced(w, force_slow_rows=variant == "slow_rows",
+                                    streaming=variant == "streaming")
+    _report(rep)
+    parity.assert_clean(rep)
+
+
+def test_degenerate_all_equal_scores_bf16():
+    """All-zero bf16 inputs through the fused routing kernel (every score ties, so every list of
+    the two-sweep kernel is one run of equal keys: all rows take its slow path): TopK must take
+    the smallest ids under the causal mask, margin 0."""
+    w = W.moderate().replace(heads=2)
+    led = RouteLedger(config_from_workload(w))
+    z = torch.zeros(1, w.problems, w.n_q, w.d, device="cuda", dtype=torch.bfloat16)
+    led.route_anchor(z, z, 0)
+    torch.cuda.synchronize()
+    assert led.status() == 0
+    r = led.routes.cpu().numpy().reshape(w.problems, w.n_q, w.k)
+    s = led.sentinels.cpu().numpy().reshape(w.problems, w.n_q, w.sw)
+    for i in (0, 5, w.k - 1, w.k, w.k + 3, w.k + w.m, 100, w.n_q - 1):
+        v = i + 1
+        kk, nn = min(w.k, v), min(w.m, max(0, v - w.k))
+        assert (np.sort(r[:, i, :kk], axis=1) == np.arange(kk)).all(), i
+        assert (r[:, i, kk:] == -1).all()
+        assert (np.sort(s[:, i, :nn], axis=1) == np.arange(kk, kk + nn)).all(), i
+        rnd = s[:, i, w.m:w.m + w.r]
+        n_rnd = min(w.r, max(0, v - kk - nn))
+        assert ((rnd >= 0).sum(axis=1) == n_rnd).all(), i
+        assert all(len(set(x[x >= 0])) == n_rnd and (x[x >= 0] >= kk + nn).all() and
+                   (x[x >= 0] < v).all() for x in rnd), i
+    mg = led.margin.cpu().numpy().reshape(w.problems, w.n_q)
+    assert (mg[:, w.k:] == 0).all() and np.isinf(mg[:, :w.k]).all()
+    assert (led.kth_score.cpu().numpy() == 0).all()
+    led.close()
+
+
 def test_ragged_shapes_and_wide_ledger():
     # n_q not a multiple of any tile, n_q != n_k, non-causal, d=64 bf16, wide candidate set
     w = W.RouteWorkload("ragged", 1, 3, 200, 333, 64, 12, 24, 12, layers=3, anchor_every=3,
