@@ -256,6 +256,7 @@ int rr_compact_flags_noalloc(const uint8_t* dev_flags, int32_t n_problems, int32
 #define RR_KIND_SCORE_TC     7   /* tcgen05 score GEMM                                       */
 #define RR_KIND_ROUTE_FUSED  8   /* tcgen05 score GEMM fused with TopK + sentinels           */
 #define RR_KIND_RESCORE_DENSE 9  /* candidate rescoring from the tensor-core score strip     */
+#define RR_KIND_SENTINELS    10  /* global + random sentinels of the rows just routed         */
 #define RR_NUM_KINDS        12
 int rr_profile_begin(rr_ledger* L);
 int rr_profile_end(rr_ledger* L, void* stream, float* total_ms, int64_t* launches);

@@ -151,6 +151,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     if (L->sweep) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer,
                                                         (L->cfg.debug_outputs >> 3) & 1, st));
+      LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, nullptr, layer, st));
     } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, nullptr, layer, st));
     } else {
@@ -168,6 +169,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     if (L->sweep) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, p.refresh_rows, layer,
                                                         (L->cfg.debug_outputs >> 3) & 1, st));
+      LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, p.refresh_rows, layer, st));
     } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
     } else {
@@ -454,6 +456,7 @@ const char* rr_kind_name(int kind) {
     case RR_KIND_SCORE_TC: return "score_tc";
     case RR_KIND_ROUTE_FUSED: return "route_fused";
     case RR_KIND_RESCORE_DENSE: return "rescore_dense";
+    case RR_KIND_SENTINELS: return "sentinels";
     default: return "";
   }
 }

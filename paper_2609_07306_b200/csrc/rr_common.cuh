@@ -117,6 +117,9 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
                                   cudaStream_t st);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
+// global + random sentinels of the listed rows (after rr_launch_route_sweep; n_k <= 1024)
+cudaError_t rr_launch_sentinels(const RRParams& p, const int32_t* row_list, int layer,
+                                cudaStream_t st);
 cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
                               cudaStream_t st);
 bool rr_rescore_dense_supported(const RRParams& p);

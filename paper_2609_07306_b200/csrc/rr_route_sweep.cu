@@ -6,7 +6,7 @@
 // One CTA owns 128 query rows of one problem (consecutive rows at an anchor; a segment of the
 // compacted refresh list at a relay, Section 4.2) and walks the key chunks in tiles of 128,
 // stopping at the last chunk any of its rows may select.
-//   warp 0     : TMA producer (Kc tiles, 128-byte swizzle, a ring of four half-tile stages, no
+//   warp 0     : TMA producer (Kc tiles, 128-byte swizzle, a ring of five half-tile stages, no
 //                multicast)
 //   warps 1, 18: one thread each issues tcgen05.mma (M=128, N=128, K=16), alternating tiles, into
 //                a ring of 3 TMEM accumulators; the Qc tile is the MMA's A operand in TMEM
@@ -26,7 +26,9 @@
 // of neighbours that agree in those bits) and writes it back in rank order.  One thread per row
 // then merges the row's four sorted lists from the top: the first k pops are the route, the
 // next m the near-miss sentinels, pop k+1 gives the margin.  Ties go to the smaller chunk id.
-// The same thread draws the random sentinels with the counter-based generator.
+// The mandatory global and the random sentinels of the routed rows are built by a separate
+// one-thread-per-row kernel (rr_sentinels.cu) that runs at full occupancy: inside this kernel,
+// which holds one CTA per SM, their serial draws would sit on every CTA's critical path.
 // Rows the fast path cannot finish exactly (a list overflowed, three or more scores agreeing in
 // 27 bits inside one list) are handed to an exact slow path: one more sweep stores their
 // complete score rows in shared memory, and a warp per row runs the radix select of the
@@ -39,7 +41,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int BM = 128, BN = 128, H_STAGES = 4, ACC_STAGES = 3;   // H_STAGES: Kc stages of one K-half
+constexpr int BM = 128, BN = 128, H_STAGES = 5, ACC_STAGES = 3;   // H_STAGES: Kc stages of one K-half
 constexpr int TPR = 4, SLICE = BN / TPR;           // threads per row, columns per thread and tile
 constexpr int SEL_WARPS = TPR * (BM / 32), ISSUE_WARPS = 2;
 constexpr int LAST_SEL = 2 + SEL_WARPS;            // warps [2, LAST_SEL) select; the second issuer follows
@@ -72,7 +74,6 @@ struct Ctl {
 };
 constexpr int CTL_BYTES = 8192;
 static_assert(sizeof(Ctl) <= CTL_BYTES, "control block too large");
-constexpr int BITMAP_BYTES = BM_WORDS * BM * 4;           // [word][row]
 constexpr int BUF_BYTES = CAPJ * ENTRY_PITCH;             // 128 KB
 static_assert(HARD_SLOTS * MAX_NK * 4 + SEL_WARPS * (256 + BM_WORDS) * 4 <= BUF_BYTES,
               "slow-path rows and per-warp scratch must fit the list area");
@@ -102,30 +103,135 @@ template <class T> struct DescF {
 template <class T> struct DescU {
   static __device__ __forceinline__ void ce(T& a, T& b) { const T hi = max(a, b), lo = min(a, b); a = hi; b = lo; }
 };
-template <int LO, int N, int R, class T, class OP> struct OEMerge {
+// LIMIT < N prunes the network to its first LIMIT inputs: valid when the inputs from LIMIT on hold
+// the smallest key and sit last, since a compare-exchange with such an input changes nothing.
+template <int LO, int N, int R, class T, class OP, int LIMIT> struct OEMerge {
   static __device__ __forceinline__ void run(T* x) {
     constexpr int M = R * 2;
     if constexpr (M < N) {
-      OEMerge<LO, N, M, T, OP>::run(x);
-      OEMerge<LO + R, N, M, T, OP>::run(x);
+      OEMerge<LO, N, M, T, OP, LIMIT>::run(x);
+      OEMerge<LO + R, N, M, T, OP, LIMIT>::run(x);
 #pragma unroll
-      for (int i = LO + R; i + R < LO + N; i += M) OP::ce(x[i], x[i + R]);
+      for (int i = LO + R; i + R < LO + N; i += M)
+        if (i + R < LIMIT) OP::ce(x[i], x[i + R]);
     } else {
-      OP::ce(x[LO], x[LO + R]);
+      if constexpr (LO + R < LIMIT) OP::ce(x[LO], x[LO + R]);
     }
   }
 };
-template <int LO, int N, class T, class OP> struct OESort {
+template <int LO, int N, class T, class OP, int LIMIT = LO + N> struct OESort {
   static __device__ __forceinline__ void run(T* x) {
-    if constexpr (N > 1) {
+    if constexpr (N > 1 && LO < LIMIT) {
       constexpr int M = N / 2;
-      OESort<LO, M, T, OP>::run(x);
-      OESort<LO + M, M, T, OP>::run(x);
-      OEMerge<LO, N, 1, T, OP>::run(x);
+      OESort<LO, M, T, OP, LIMIT>::run(x);
+      OESort<LO + M, M, T, OP, LIMIT>::run(x);
+      OEMerge<LO, N, 1, T, OP, LIMIT>::run(x);
     }
   }
 };
 
+// ---- sorting one list of sweep 2 ------------------------------------------------------------
+// The list (n <= LIMIT <= 32 entries {score, id} at base + e * ENTRY_PITCH, in ascending chunk id)
+// is rewritten in rank order (score descending, id ascending).  Keys = 27 score bits | (31 -
+// position), sorted by a network in registers; neighbours that agree in the 27 bits are ordered
+// by position at that point and are repaired with the exact scores (equal scores keep the
+// position order = ascending chunk id); three in a row are reported (slow path).
+template <int LIMIT>
+__device__ __forceinline__ bool sort_list(uint32_t base, int n) {
+  uint32_t key[CAPJ];
+#pragma unroll
+  for (int e = 0; e < CAPJ; ++e) {
+    key[e] = 0u;
+    if (e < LIMIT) {
+      uint32_t sb;
+      asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sb) : "r"(base + (uint32_t)e * ENTRY_PITCH) : "memory");
+      const uint32_t ok = rr_order_key(__uint_as_float(sb));
+      key[e] = e < n ? ((ok & ~31u) | (uint32_t)(31 - e)) : 0u;
+    }
+  }
+  OESort<0, CAPJ, uint32_t, DescU<uint32_t>, LIMIT>::run(key);
+  bool same = false, run3 = false;
+#pragma unroll
+  for (int i = 0; i + 1 < LIMIT; ++i) same |= key[i + 1] >= 32u && ((key[i] ^ key[i + 1]) < 32u);
+  if (__any_sync(0xFFFFFFFFu, same)) {
+#pragma unroll
+    for (int i = 0; i + 1 < LIMIT; ++i) {
+      const bool pair = key[i + 1] >= 32u && ((key[i] ^ key[i + 1]) < 32u);
+      if (pair) {
+        uint32_t sa, sb;
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sa) : "r"(base + (31u - (key[i] & 31u)) * ENTRY_PITCH) : "memory");
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sb) : "r"(base + (31u - (key[i + 1] & 31u)) * ENTRY_PITCH) : "memory");
+        if (__uint_as_float(sb) > __uint_as_float(sa)) { const uint32_t t = key[i]; key[i] = key[i + 1]; key[i + 1] = t; }
+        if (i + 2 < LIMIT && key[i + 2] >= 32u && ((key[i] ^ key[i + 2]) < 32u)) run3 = true;
+      }
+    }
+  }
+  // write the list back in rank order: all loads first, then all stores
+  uint32_t es[LIMIT], ei[LIMIT];
+#pragma unroll
+  for (int i = 0; i < LIMIT; ++i)
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(es[i]), "=r"(ei[i])
+                 : "r"(base + (31u - (key[i] & 31u)) * ENTRY_PITCH) : "memory");
+#pragma unroll
+  for (int i = 0; i < LIMIT; ++i)
+    if (i < n) asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(base + (uint32_t)i * ENTRY_PITCH), "r"(es[i]), "r"(ei[i]) : "memory");
+  return run3;
+}
+
+
+// ---- exchange selection over four sorted lists -----------------------------------------------
+// The four lists of a row (scores in descending order in the score words of its list entries,
+// n_j entries each) and a split a_0 + a_1 + a_2 + a_3 = T: the first a_j entries of list j are
+// "in".  One entry at a time leaves the list whose last entry in is the smallest and one enters
+// from the list whose first entry out is the largest, while the latter is larger; every such
+// move raises the sum of what is in, so the search ends, and it ends at the split that holds the
+// T largest scores: lo = the smallest score in (the T-th largest), hi = the largest score out.
+// Any split reached on the way already has T scores at or above its lo.
+// Two entries on either side of each cut are kept in registers, so a move is a register shuffle
+// and its refill load has a full step to arrive.  Warp-uniform: lanes that are done idle.
+struct Exchange { int a0, a1, a2, a3; float lo, hi; };
+__device__ __forceinline__ float exch_score(uint32_t row_base, int j, int e, int nj) {
+  uint32_t bits;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(bits)
+               : "r"(row_base + (uint32_t)j * LIST_PITCH + (uint32_t)min(max(e, 0), CAPJ - 1) * ENTRY_PITCH)
+               : "memory");
+  return e < 0 ? __int_as_float(0x7f800000) : (e >= nj ? __int_as_float(0xff800000) : __uint_as_float(bits));
+}
+__device__ __forceinline__ Exchange exchange_select(uint32_t row_base, int n0, int n1, int n2, int n3,
+                                                    int a0, int a1, int a2, int a3, bool on,
+                                                    int max_steps) {
+  const float ninf = __int_as_float(0xff800000);
+#define RR_WIN(j) \
+  float p##j = exch_score(row_base, j, a##j - 2, n##j), l##j = exch_score(row_base, j, a##j - 1, n##j), \
+        x##j = exch_score(row_base, j, a##j, n##j), y##j = exch_score(row_base, j, a##j + 1, n##j);
+  RR_WIN(0) RR_WIN(1) RR_WIN(2) RR_WIN(3)
+#undef RR_WIN
+  float lo = fminf(fminf(l0, l1), fminf(l2, l3)), hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+  for (int it = 0; it < max_steps; ++it) {
+    const int jm = l0 == lo ? 0 : l1 == lo ? 1 : l2 == lo ? 2 : 3;
+    const float z0 = jm == 0 ? ninf : x0, z1 = jm == 1 ? ninf : x1;
+    const float z2 = jm == 2 ? ninf : x2, z3 = jm == 3 ? ninf : x3;
+    const float hz = fmaxf(fmaxf(z0, z1), fmaxf(z2, z3));
+    const int jx = z0 == hz ? 0 : z1 == hz ? 1 : z2 == hz ? 2 : 3;
+    const bool move = on && hz > lo;
+    if (!__any_sync(0xFFFFFFFFu, move)) break;
+    // refills: the entry two before the new cut of jm, the entry one behind the new cut of jx
+    const int am = jm == 0 ? a0 : jm == 1 ? a1 : jm == 2 ? a2 : a3;
+    const int ax = jx == 0 ? a0 : jx == 1 ? a1 : jx == 2 ? a2 : a3;
+    const int nx = jx == 0 ? n0 : jx == 1 ? n1 : jx == 2 ? n2 : n3;
+    const float rp = exch_score(row_base, jm, am - 3, CAPJ), ry = exch_score(row_base, jx, ax + 2, nx);
+    if (move) {
+#define RR_MOVE(j) \
+      if (jm == j) { y##j = x##j; x##j = l##j; l##j = p##j; p##j = rp; --a##j; } \
+      if (jx == j) { p##j = l##j; l##j = x##j; x##j = y##j; y##j = ry; ++a##j; }
+      RR_MOVE(0) RR_MOVE(1) RR_MOVE(2) RR_MOVE(3)
+#undef RR_MOVE
+    }
+    lo = fminf(fminf(l0, l1), fminf(l2, l3));
+    hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+  }
+  return Exchange{a0, a1, a2, a3, lo, hi};
+}
 
 // ---- threshold filter of sweep 2 ------------------------------------------------------------
 // One score: if it passes, {score, chunk id} goes to [w] and w moves on by one entry.  Written in
@@ -180,13 +286,13 @@ template <int I0>
 __device__ __forceinline__ void filter_group(uint32_t& w, const uint32_t (&acc)[SLICE], float tau,
                                              uint32_t col0, uint32_t v, uint32_t w_end, bool inner) {
   const bool tight = __any_sync(0xFFFFFFFFu, w + 8u * ENTRY_PITCH > w_end);
+  (void)inner;
   if (tight) filter_eight<I0, true, true>(w, acc, tau, col0, v, w_end);
-  else if (inner) filter_eight<I0, false, false>(w, acc, tau, col0, v, w_end);
   else filter_eight<I0, true, false>(w, acc, tau, col0, v, w_end);
 }
 
 #ifdef RR_PHASE_TIMING
-__device__ unsigned long long g_sweep_phase[16];
+__device__ unsigned long long g_sweep_phase[32];
 #define PH_T0() long long ph_t0_ = clock64()
 #define PH_LAP(i) do { const long long t1_ = clock64(); if ((threadIdx.x & 31) == 0) atomicAdd(&g_sweep_phase[i], (unsigned long long)(t1_ - ph_t0_)); ph_t0_ = t1_; } while (0)
 #define PH_CNT(i, val_) atomicAdd(&g_sweep_phase[i], (unsigned long long)(val_))
@@ -200,16 +306,18 @@ template <int D>
 __global__ void __launch_bounds__(NT, 1)
 route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
-                   uint32_t layer, int quota, int force_hard) {
+                   uint32_t layer, int quota, int qstep, int force_hard) {
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sB = smem;
   Ctl* ctl = (Ctl*)(smem + H_STAGES * C::B_HALF);
-  uint8_t* s_bitmap = (uint8_t*)ctl + CTL_BYTES;
-  uint8_t* s_buf = s_bitmap + BITMAP_BYTES;
+  uint8_t* s_buf = (uint8_t*)ctl + CTL_BYTES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef RR_PHASE_TIMING
+  const long long cta_t0_ = clock64();
+#endif
   // Row tiles are handed out heaviest first (under the causal mask the last tile of a problem
   // walks the most key chunks), so the tail of the grid is made of the short ones.
   const int tiles_m = p.tiles_per_problem;
@@ -219,15 +327,39 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   if (row_list) { seg_lo = p.problem_offsets[prob]; seg_hi = p.problem_offsets[prob + 1]; }
   if (tm * BM >= seg_hi - seg_lo) return;                 // nothing to do (uniform per CTA)
 
-  if (tid < BM) {
-    const int local = tm * BM + tid;
-    int row = -1, slot = 0;
+  // row of the CTA's tile -> query row of the problem and its slot (position in the refresh list,
+  // or global row id); -1 = no row
+  auto locate = [&](int rr, int& row_out, int& slot_out) {
+    const int local = tm * BM + rr;
+    row_out = -1; slot_out = 0;
     if (row_list) {
       const int s = seg_lo + local;
-      if (s < seg_hi) { row = row_list[s] - prob * p.n_q; slot = s; }
+      if (s < seg_hi) { row_out = row_list[s] - prob * p.n_q; slot_out = s; }
     } else if (local < p.n_q) {
-      row = local; slot = prob * p.n_q + local;
+      row_out = local; slot_out = prob * p.n_q + local;
     }
+  };
+  // ---- the Qc tile goes to TMEM: the first thread of row r loads the row (two bf16 per 32-bit
+  // word, as they lie in memory; refresh rows are not contiguous, so this is also the gather)
+  // and stores it to TMEM lane r, where the MMA reads its A operand; rows without a query are 0.
+  // The loads are issued first so that their latency overlaps the rest of the set-up.
+  constexpr int QW = D / 2;                                // 32-bit words per row
+  uint32_t qv[QW];
+  const bool q_loader = warp >= 2 && warp < 6;
+  if (q_loader) {
+    int qrow, qslot;
+    locate((warp & 3) * 32 + lane, qrow, qslot);
+    const uint4* src = reinterpret_cast<const uint4*>(qc + ((size_t)prob * p.n_q + max(qrow, 0)) * D);
+#pragma unroll
+    for (int i = 0; i < QW / 4; ++i) {
+      uint4 t = make_uint4(0, 0, 0, 0);
+      if (qrow >= 0) t = __ldg(src + i);
+      qv[4 * i] = t.x; qv[4 * i + 1] = t.y; qv[4 * i + 2] = t.z; qv[4 * i + 3] = t.w;
+    }
+  }
+  if (tid < BM) {
+    int row, slot;
+    locate(tid, row, slot);
     ctl->row[tid] = row; ctl->slot[tid] = slot;
     ctl->hard_slot[tid] = -1;
   }
@@ -243,26 +375,12 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     tma_prefetch_desc(&tmap_k);
   }
   if (warp == 0) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+  tc_fence_before();
   __syncthreads();
-
-  // ---- the Qc tile goes to TMEM: the first thread of row r loads the row (two bf16 per 32-bit
-  // word, as they lie in memory; refresh rows are not contiguous, so this is also the gather)
-  // and stores it to TMEM lane r, where the MMA reads its A operand; rows without a query are 0
   tc_fence_after();
-  if (warp >= 2 && warp < 6) {
-    const int r = (warp & 3) * 32 + lane;
-    const int row = ctl->row[r];
-    constexpr int W = D / 2;                               // 32-bit words per row
-    uint32_t qv[W];
-    const uint4* src = reinterpret_cast<const uint4*>(qc + ((size_t)prob * p.n_q + max(row, 0)) * D);
-#pragma unroll
-    for (int i = 0; i < W / 4; ++i) {
-      uint4 t = make_uint4(0, 0, 0, 0);
-      if (row >= 0) t = __ldg(src + i);
-      qv[4 * i] = t.x; qv[4 * i + 1] = t.y; qv[4 * i + 2] = t.z; qv[4 * i + 3] = t.w;
-    }
+  if (q_loader) {
     const uint32_t taddr = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_COL;
-    if constexpr (W == 64) tmem_st_32x64(taddr, qv); else tmem_st_32x32(taddr, qv);
+    if constexpr (QW == 64) tmem_st_32x64(taddr, qv); else tmem_st_32x32(taddr, qv);
     tmem_st_wait();
   }
   tc_fence_before();
@@ -360,7 +478,6 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   const uint32_t buf0 = smem_u32(s_buf);
   const uint32_t row_base = buf0 + (uint32_t)r * 8u;                       // list 0, entry 0
   const uint32_t my_base = row_base + (uint32_t)jslice * LIST_PITCH;       // this thread's list
-  const uint32_t bm_row = smem_u32(s_bitmap) + (uint32_t)r * 4u;           // word w at + w*BM*4
   const uint32_t acc_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(jslice * SLICE);
   int vmaxw = v, vminw = row >= 0 ? v : 0x7FFFFFFF;
 #pragma unroll
@@ -375,7 +492,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   auto tile_wait = [&](int gt) -> int {
     const int as = gt % ACC_STAGES; const uint32_t aph = (gt / ACC_STAGES) & 1;
     if (alive) {
-      const bool ready = mbar_wait_warp(&ctl->acc_full[as], aph, abort_flag, 64);
+      const bool ready = mbar_wait_warp(&ctl->acc_full[as], aph, abort_flag, 20);
       if (!__all_sync(FULL, ready)) alive = false;
     }
     if (!alive) return -1;
@@ -407,6 +524,9 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     __syncwarp();
   } else {
     PH_T0();
+#ifdef RR_PHASE_TIMING
+    if (lane == 0) PH_CNT(7, ph_t0_ - cta_t0_);
+#endif
     // ===== sweep 1: group maxima -> tau ==========================================================
     float mx[SLICE];
 #pragma unroll
@@ -428,62 +548,48 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       tile_release(t);
     }
     PH_LAP(0);
-    OESort<0, SLICE, float, DescF<float>>::run(mx);
-    // The row's keep-th largest group maximum (over the 128 groups of its four threads) is the
-    // tightest bound the maxima give.  Each thread publishes its sorted maxima in the score words
-    // of its (still empty) list; every thread of the row then finds how many maxima each list
-    // contributes to the top keep: starting from an even split it moves one unit of quota at a
-    // time from the list whose last contributing maximum is the smallest to the list whose next
-    // maximum is the largest, while that next maximum is the larger of the two.  Every split
-    // with quotas adding up to keep gives a valid bound (keep distinct scores lie at or above
-    // the smallest contributing maximum), so stopping early is safe.  Rows that fit one tile
-    // keep everything (their lists cannot overflow).
+#ifdef RR_LOCKSTEP
+    asm volatile("bar.sync 5, 512;" ::: "memory");
+    PH_LAP(14);
+#endif
+    OESort<0, SLICE, float, DescF<float>, SLICE>::run(mx);
+#ifdef RR_ICACHE_PROBE
+    PH_LAP(11);
+    // the same code again on a copy (a value the compiler cannot know keeps it from folding)
+    for (int rep_ = 0; rep_ < 2; ++rep_) {
+      float my[SLICE];
+#pragma unroll
+      for (int i = 0; i < SLICE; ++i) my[i] = mx[(i * 7) & 31] + (float)(quota >> 20);
+      OESort<0, SLICE, float, DescF<float>, SLICE>::run(my);
+      if (my[0] < my[31]) mx[0] = my[5];
+      if (rep_ == 0) PH_LAP(12); else PH_LAP(13);
+    }
+#endif
+    // The row's keep-th largest group maximum (over the 128 groups of its four threads) has keep
+    // distinct scores of the row at or above it: a valid inclusive lower bound of the row's
+    // keep-th largest score, and the tightest one the maxima give (about 1.2 keep scores pass;
+    // an even split of keep over the four threads would let 1.5 keep pass, and lists overflow).
+    // Each thread publishes its sorted maxima in the score words of its (still empty) list; the
+    // first thread of the row finds the split by exchange (exchange_select).  Rows that fit one
+    // tile keep everything (their lists cannot overflow).
 #pragma unroll
     for (int i = 0; i < SLICE; ++i) sts32(my_base + (uint32_t)i * ENTRY_PITCH, __float_as_uint(mx[i]));
+    PH_LAP(8);
     quarter_sync(quarter);
+    PH_LAP(9);
     float tau = ninf;
     if (jslice == 0) {          // one thread per row searches; the others wait at the barrier
       const int keep_cfg_ = p.k + max(p.m, 1);
       const bool bounded = row >= 0 && v >= BN;              // v >= 128 > keep: all 128 groups exist
-      auto mxat = [&](int j, int a) -> float {               // a-th largest maximum of list j (1-based)
-        const float val = __uint_as_float(lds32(row_base + (uint32_t)j * LIST_PITCH +
-                                                (uint32_t)min(max(a - 1, 0), SLICE - 1) * ENTRY_PITCH));
-        return a < 1 ? pinf : (a > SLICE ? ninf : val);
-      };
-      int a0 = keep_cfg_ / TPR + (0 < keep_cfg_ % TPR), a1 = keep_cfg_ / TPR + (1 < keep_cfg_ % TPR);
-      int a2 = keep_cfg_ / TPR + (2 < keep_cfg_ % TPR), a3 = keep_cfg_ / TPR;
-      float l0 = mxat(0, a0), l1 = mxat(1, a1), l2 = mxat(2, a2), l3 = mxat(3, a3);       // last in
-      float x0 = mxat(0, a0 + 1), x1 = mxat(1, a1 + 1), x2 = mxat(2, a2 + 1), x3 = mxat(3, a3 + 1);  // next out
-      for (int it = 0; it < MAX_KEEP; ++it) {
-        const float lo = fminf(fminf(l0, l1), fminf(l2, l3));
-        const int jm = l0 == lo ? 0 : l1 == lo ? 1 : l2 == lo ? 2 : 3;
-        const float y0 = jm == 0 ? ninf : x0, y1 = jm == 1 ? ninf : x1;
-        const float y2 = jm == 2 ? ninf : x2, y3 = jm == 3 ? ninf : x3;
-        const float hi = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
-        const int jx = y0 == hi ? 0 : y1 == hi ? 1 : y2 == hi ? 2 : 3;
-        const bool move = bounded && hi > lo;
-        if (!__any_sync(FULL, move)) break;
-        // list jm gives up its last maximum, list jx takes in its next one
-        const int am = (jm == 0 ? a0 : jm == 1 ? a1 : jm == 2 ? a2 : a3) - 1;
-        const int ax = (jx == 0 ? a0 : jx == 1 ? a1 : jx == 2 ? a2 : a3) + 1;
-        const float lm = mxat(jm, am), xx = mxat(jx, ax + 1);
-        if (move) {
-          x0 = jm == 0 ? l0 : x0; x1 = jm == 1 ? l1 : x1; x2 = jm == 2 ? l2 : x2; x3 = jm == 3 ? l3 : x3;
-          l0 = jm == 0 ? lm : l0; l1 = jm == 1 ? lm : l1; l2 = jm == 2 ? lm : l2; l3 = jm == 3 ? lm : l3;
-          l0 = jx == 0 ? x0 : l0; l1 = jx == 1 ? x1 : l1; l2 = jx == 2 ? x2 : l2; l3 = jx == 3 ? x3 : l3;
-          x0 = jx == 0 ? xx : x0; x1 = jx == 1 ? xx : x1; x2 = jx == 2 ? xx : x2; x3 = jx == 3 ? xx : x3;
-          a0 += (jx == 0) - (jm == 0); a1 += (jx == 1) - (jm == 1);
-          a2 += (jx == 2) - (jm == 2); a3 += (jx == 3) - (jm == 3);
-        }
-      }
-      if (bounded) tau = fminf(fminf(l0, l1), fminf(l2, l3));
+      const int q_ = keep_cfg_ / TPR, rm_ = keep_cfg_ % TPR;
+      const Exchange ex = exchange_select(row_base, SLICE, SLICE, SLICE, SLICE, q_ + (0 < rm_),
+                                          q_ + (1 < rm_), q_ + (2 < rm_), q_, bounded, MAX_KEEP);
+      if (bounded) tau = ex.lo;
       ctl->tau_row[r] = tau;
     }
+    PH_LAP(10);
     quarter_sync(quarter);                  // the published maxima have been read: lists are free
     tau = ctl->tau_row[r];
-    // the row's exclusion bitmap is cleared by its four threads, eight words each
-#pragma unroll
-    for (int w = 0; w < BM_WORDS / TPR; ++w) sts32(bm_row + (uint32_t)(jslice * (BM_WORDS / TPR) + w) * (BM * 4u), 0u);
     // rows of a refresh list also have the bound the rescoring kernel derived from the old
     // candidates' current scores (bit-identical scores: no margin needed)
     if (row_list && row >= 0) tau = fmaxf(tau, p.tau[g]);
@@ -511,47 +617,23 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     bool slow = n_raw > CAPJ;                              // the list overflowed
     const int n = min(n_raw, CAPJ);
 
-    // ===== sort the list: keys = 27 score bits | (31 - position) ================================
-    uint32_t key[CAPJ];
-#pragma unroll
-    for (int e = 0; e < CAPJ; ++e) {
-      const uint32_t sb = lds32(my_base + (uint32_t)e * ENTRY_PITCH);
-      const uint32_t ok = rr_order_key(__uint_as_float(sb));
-      key[e] = e < n ? ((ok & ~31u) | (uint32_t)(31 - e)) : 0u;
-    }
-    OESort<0, CAPJ, uint32_t, DescU<uint32_t>>::run(key);
-    // neighbours that agree in the 27 bits are ordered by position so far: repair them with
-    // the exact scores (equal scores keep the position order = ascending chunk id); three in
-    // a row are left to the slow path
-    bool same = false;
-#pragma unroll
-    for (int i = 0; i + 1 < CAPJ; ++i) same |= key[i + 1] >= 32u && ((key[i] ^ key[i + 1]) < 32u);
-    if (__any_sync(FULL, same)) {
-#pragma unroll
-      for (int i = 0; i + 1 < CAPJ; ++i) {
-        const bool pair = key[i + 1] >= 32u && ((key[i] ^ key[i + 1]) < 32u);
-        if (pair) {
-          const float sa = __uint_as_float(lds32(my_base + (31u - (key[i] & 31u)) * ENTRY_PITCH));
-          const float sb = __uint_as_float(lds32(my_base + (31u - (key[i + 1] & 31u)) * ENTRY_PITCH));
-          if (sb > sa) { const uint32_t t = key[i]; key[i] = key[i + 1]; key[i + 1] = t; }
-          if (i + 2 < CAPJ && key[i + 2] >= 32u && ((key[i] ^ key[i + 2]) < 32u)) slow = true;
-        }
-      }
-    }
-    // write the list back in rank order: all loads first, then all stores
+    // ===== sort the list (network sized for the longest list of the warp) =========================
+#ifdef RR_LOCKSTEP
+    asm volatile("bar.sync 5, 512;" ::: "memory");
+    PH_LAP(15);
+#endif
     {
-      uint32_t es[CAPJ], ei[CAPJ];
-#pragma unroll
-      for (int i = 0; i < CAPJ; ++i)
-        lds64(my_base + (31u - (key[i] & 31u)) * ENTRY_PITCH, es[i], ei[i]);
-#pragma unroll
-      for (int i = 0; i < CAPJ; ++i)
-        if (i < n) sts64(my_base + (uint32_t)i * ENTRY_PITCH, es[i], ei[i]);
+      const int n_warp = __reduce_max_sync(FULL, n);
+      bool run3;
+      if (n_warp <= 16) run3 = sort_list<16>(my_base, n);
+      else if (n_warp <= 24) run3 = sort_list<24>(my_base, n);
+      else run3 = sort_list<32>(my_base, n);
+      slow |= run3;
     }
 #ifdef RR_PHASE_COUNTS
-    if (row >= 0 && n_raw > CAPJ) PH_CNT(9, 1);
-    if (row >= 0 && slow && n_raw <= CAPJ) PH_CNT(10, 1);
-    if (row >= 0) { PH_CNT(11, n_raw); PH_CNT(12, 1); }
+    if (row >= 0 && n_raw > CAPJ) PH_CNT(17, 1);
+    if (row >= 0 && slow && n_raw <= CAPJ) PH_CNT(18, 1);
+    if (row >= 0) { PH_CNT(22, n_raw); PH_CNT(23, 1); }
 #endif
     if (force_hard && row >= 0 && g % 5 == 0) slow = true;     // test hook: exercise the slow path
     ctl->cnt[jslice][r] = (uint32_t)n | (slow ? 256u : 0u);
@@ -576,11 +658,6 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     if (jslice < 2 && (jslice == 0 || p.m > 0)) {
       const int T = jslice == 0 ? kk0 : keep_row0;
       const int n0 = (int)(c0 & 255u), n1 = (int)(c1 & 255u), n2 = (int)(c2 & 255u), n3 = (int)(c3 & 255u);
-      auto score_at = [&](int j, int e, int nj) -> float {      // e-th entry (0-based) of list j
-        const float sc = __uint_as_float(lds32(row_base + (uint32_t)j * LIST_PITCH +
-                                               (uint32_t)min(max(e, 0), CAPJ - 1) * ENTRY_PITCH));
-        return e < 0 ? pinf : (e >= nj ? ninf : sc);
-      };
       const int nt = max(n_total, 1);
       int a0 = T * n0 / nt, a1 = T * n1 / nt, a2 = T * n2 / nt, a3 = T * n3 / nt;
       int rem = T - (a0 + a1 + a2 + a3);
@@ -591,37 +668,17 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         if (rem > 0 && a2 < n2) { ++a2; --rem; }
         if (rem > 0 && a3 < n3) { ++a3; --rem; }
       }
-      float l0 = score_at(0, a0 - 1, n0), l1 = score_at(1, a1 - 1, n1), l2 = score_at(2, a2 - 1, n2), l3 = score_at(3, a3 - 1, n3);
-      float x0 = score_at(0, a0, n0), x1 = score_at(1, a1, n1), x2 = score_at(2, a2, n2), x3 = score_at(3, a3, n3);
-      float lo = pinf, hi = ninf;
-      for (int it = 0; it <= 2 * MAX_KEEP; ++it) {
-        lo = fminf(fminf(l0, l1), fminf(l2, l3));
-        const int jm = l0 == lo ? 0 : l1 == lo ? 1 : l2 == lo ? 2 : 3;
-        const float y0 = jm == 0 ? ninf : x0, y1 = jm == 1 ? ninf : x1;
-        const float y2 = jm == 2 ? ninf : x2, y3 = jm == 3 ? ninf : x3;
-        const float hy = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
-        hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-        const int jx = y0 == hy ? 0 : y1 == hy ? 1 : y2 == hy ? 2 : 3;
-        const bool move = T > 0 && hy > lo;
-        if (!__any_sync(FULL, move)) break;
-        const int am = (jm == 0 ? a0 : jm == 1 ? a1 : jm == 2 ? a2 : a3) - 1;    // new count of jm
-        const int ax = (jx == 0 ? a0 : jx == 1 ? a1 : jx == 2 ? a2 : a3) + 1;    // new count of jx
-        const int nx = jx == 0 ? n0 : jx == 1 ? n1 : jx == 2 ? n2 : n3;
-        const float lm = score_at(jm, am - 1, CAPJ), xx = score_at(jx, ax, nx);
-        if (move) {
-          x0 = jm == 0 ? l0 : x0; x1 = jm == 1 ? l1 : x1; x2 = jm == 2 ? l2 : x2; x3 = jm == 3 ? l3 : x3;
-          l0 = jm == 0 ? lm : l0; l1 = jm == 1 ? lm : l1; l2 = jm == 2 ? lm : l2; l3 = jm == 3 ? lm : l3;
-          l0 = jx == 0 ? x0 : l0; l1 = jx == 1 ? x1 : l1; l2 = jx == 2 ? x2 : l2; l3 = jx == 3 ? x3 : l3;
-          x0 = jx == 0 ? xx : x0; x1 = jx == 1 ? xx : x1; x2 = jx == 2 ? xx : x2; x3 = jx == 3 ? xx : x3;
-          a0 += (jx == 0) - (jm == 0); a1 += (jx == 1) - (jm == 1);
-          a2 += (jx == 2) - (jm == 2); a3 += (jx == 3) - (jm == 3);
-        }
-      }
+      const Exchange ex = exchange_select(row_base, n0, n1, n2, n3, a0, a1, a2, a3, T > 0, 2 * MAX_KEEP + 1);
+      a0 = ex.a0; a1 = ex.a1; a2 = ex.a2; a3 = ex.a3;
+      const float lo = ex.lo, hi = ex.hi;
       // not settled: scores tie across the cut, or the exchange ran out of steps
       const bool unsettled = T > 0 && !(lo > hi);
       const uint32_t cut4 = (uint32_t)a0 | ((uint32_t)a1 << 8) | ((uint32_t)a2 << 16) | ((uint32_t)a3 << 24);
       if (jslice == 0) { ctl->cut_k[r] = cut4; ctl->cut_bad[0][r] = unsettled; kth = lo; next = hi; }
       else { ctl->cut_keep[r] = cut4; ctl->cut_bad[1][r] = unsettled; }
+#ifdef RR_PHASE_COUNTS
+      if (unsettled) PH_CNT(19 + jslice, 1);
+#endif
     }
     PH_LAP(4);
     quarter_sync(quarter);
@@ -647,32 +704,20 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       off_k += j < jslice ? ckj : 0;
       off_n += j < jslice ? cdj - ckj : 0;
     }
-    uint32_t idr[CAPJ];
-    const int my_d_max = __reduce_max_sync(FULL, my_d);
-#pragma unroll
-    for (int e0 = 0; e0 < CAPJ; e0 += 8) {
-      if (e0 < my_d_max) {
-#pragma unroll
-        for (int e = e0; e < e0 + 8; ++e) idr[e] = lds32(my_base + (uint32_t)e * ENTRY_PITCH + 4u);
-      }
-    }
-    quarter_sync(quarter);                 // every list of the row has been read: its space is free
-    // staging area of a row = the 64 words of its first list: route ids in words [0, k), near-miss
-    // ids in [k, k+m); set bits of the exclusion bitmap on the way
-    auto stage_addr = [&](int o) -> uint32_t {
-      return row_base + (uint32_t)(o >> 1) * ENTRY_PITCH + (uint32_t)(o & 1) * 4u;
-    };
-#pragma unroll
-    for (int e0 = 0; e0 < CAPJ; e0 += 8) {
-      if (e0 < my_d_max) {
-#pragma unroll
-        for (int e = e0; e < e0 + 8; ++e) {
-          if (e < my_d) {
-            const int o = e < my_k ? off_k + e : p.k + off_n + (e - my_k);
-            sts32(stage_addr(o), idr[e]);
-            asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(bm_row + (idr[e] >> 5) * (BM * 4u)),
-                         "r"(1u << (idr[e] & 31u)) : "memory");
-          }
+    // staging area of the CTA's outputs = the Kc ring (idle once the last tile of sweep 2 has
+    // been consumed; the slow path only starts behind the CTA-wide barrier): word o of row r at
+    // [o][r]; route ids in words [0, k), near-miss ids in [k, k+m).  Each thread moves the ids of
+    // its own entries.
+    const uint32_t stage_row = smem_u32(sB) + (uint32_t)r * 4u;
+    auto stage_addr = [&](int o) -> uint32_t { return stage_row + (uint32_t)o * (BM * 4u); };
+    {
+      const int my_d_max = __reduce_max_sync(FULL, my_d);
+#pragma unroll 1
+      for (int e = 0; e < my_d_max; ++e) {
+        if (e < my_d) {
+          const uint32_t id = lds32(my_base + (uint32_t)e * ENTRY_PITCH + 4u);
+          const int o = e < my_k ? off_k + e : p.k + off_n + (e - my_k);
+          sts32(stage_addr(o), id);
         }
       }
     }
@@ -700,82 +745,11 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
         }
       }
     }
-    // ---- random sentinels, part 1: the first 32 draws of the row's sequence, eight per thread,
-    // into the (free) second list of the row; they do not depend on what is excluded
-    auto draw_addr = [&](int t) -> uint32_t {
-      return row_base + LIST_PITCH + (uint32_t)(t >> 1) * ENTRY_PITCH + (uint32_t)(t & 1) * 4u;
-    };
-    const bool sample = go && p.r > 0 && v - (kk + n_near) > p.r;    // else the whole pool is taken
-    const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
-    if (__any_sync(FULL, sample)) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int t = jslice * 8 + i;
-        sts32(draw_addr(t), __umulhi(rr_draw_u32(rk, layer, (uint32_t)t), (uint32_t)v));
-      }
-    }
-    PH_LAP(5);
-    quarter_sync(quarter);
     if (jslice == 0 && go) {
       p.kth[g] = kth;
       p.margin[g] = v > kk ? kth - next : pinf;
-      int32_t* sent = p.sentinels + (size_t)g * p.sw;
-      auto bm = [&](int w) -> uint32_t { return bm_row + (uint32_t)w * (BM * 4u); };
-      // ---- mandatory global sentinels (sink chunk, most recent chunk): a slot each after
-      // the random ones, empty if the chunk is already in the route or a near-miss sentinel
-      int pool = v - (kk + n_near);
-      if (p.n_global) {
-        int32_t* glob = sent + p.m + p.r;
-        int gi = 0;
-        for (int b = 0; b < 2; ++b) {
-          if (!((p.global_mask >> b) & 1)) continue;
-          const int j = b == 0 ? 0 : v - 1;
-          int id = -1;
-          if (v > 0) {
-            const uint32_t wa = bm(j >> 5);
-            const uint32_t w = lds32(wa), bit = 1u << (j & 31);
-            if (!(w & bit)) { sts32(wa, w | bit); id = j; --pool; }
-          }
-          glob[gi++] = id;
-        }
-      }
-      // ---- random sentinels, part 2: accept strictly in draw order --------------------------
-      int32_t* rnd = sent + p.m;
-      int taken = 0;
-      if (p.r > 0 && pool > 0) {
-        if (pool > p.r) {
-          const int limit = 64 * p.r;
-          int t = 0;
-          if (sample) {                       // the draws the row's threads prepared
-            for (; t < 32 && t < limit && taken < p.r; ++t) {
-              const int j = (int)lds32(draw_addr(t));
-              const uint32_t wa = bm(j >> 5);
-              const uint32_t w = lds32(wa), bit = 1u << (j & 31);
-              if (!(w & bit)) { sts32(wa, w | bit); rnd[taken++] = j; }
-            }
-          }
-          // beyond them (many rejections: small pools), four draws at a time
-          for (int t0 = t; t0 < limit && taken < p.r; t0 += 4) {
-            int j4[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              j4[i] = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)(t0 + i)), (uint32_t)v);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const bool live = (t0 + i < limit) & (taken < p.r);
-              const uint32_t wa = bm(j4[i] >> 5);
-              const uint32_t w = lds32(wa), bit = 1u << (j4[i] & 31);
-              const bool take = live & ((w & bit) == 0u);
-              if (take) { sts32(wa, w | bit); rnd[taken] = j4[i]; }
-              taken += take;
-            }
-          }
-        }
-        for (int j = 0; j < v && taken < p.r; ++j)
-          if (!((lds32(bm(j >> 5)) >> (j & 31)) & 1u)) rnd[taken++] = j;
-      }
-      for (int e = taken; e < p.r; ++e) rnd[e] = -1;
     }
+    PH_LAP(5);
     PH_LAP(6);
   }
 
@@ -784,7 +758,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   // keys) over the list area; a warp per row then runs the exact radix select on them.
   __syncthreads();
   const int n_hard = ctl->abort_flag ? 0 : (int)ctl->hard_n;
-  if (tid == 0) { PH_CNT(8, n_hard); PH_CNT(13, n_hard > 0 ? 1 : 0); }
+  if (tid == 0) { PH_CNT(16, n_hard); PH_CNT(21, n_hard > 0 ? 1 : 0); }
   int next_gt = 2 * n_tiles;
   for (int done = 0; done < n_hard; done += HARD_SLOTS) {
     // barrier: the previous batch's rows and scratch are free again; the vote makes the
@@ -832,6 +806,9 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 
   tc_fence_before();
   __syncthreads();
+#ifdef RR_PHASE_TIMING
+  if (tid == 0) { PH_CNT(14, clock64() - cta_t0_); PH_CNT(15, 1); }
+#endif
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
@@ -841,17 +818,17 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 
 size_t smem_bytes(int d) {
   (void)d;
-  return 1024 + (size_t)H_STAGES * BN * 128 + CTL_BYTES + BITMAP_BYTES + BUF_BYTES;
+  return 1024 + (size_t)H_STAGES * BN * 128 + CTL_BYTES + BUF_BYTES;
 }
 
 }  // namespace
 
 #ifdef RR_PHASE_TIMING
-extern "C" int rr_debug_sweep_phase_counters(unsigned long long* out16, int reset) {
+extern "C" int rr_debug_sweep_phase_counters(unsigned long long* out32, int reset) {
   cudaDeviceSynchronize();
-  if (cudaMemcpyFromSymbol(out16, g_sweep_phase, sizeof(unsigned long long) * 16) != cudaSuccess) return -1;
+  if (cudaMemcpyFromSymbol(out32, g_sweep_phase, sizeof(unsigned long long) * 32) != cudaSuccess) return -1;
   if (reset) {
-    unsigned long long z[16] = {};
+    unsigned long long z[32] = {};
     cudaMemcpyToSymbol(g_sweep_phase, z, sizeof z);
   }
   return 0;
@@ -877,6 +854,7 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
   const int grid = p.P * p.tiles_per_problem;
   const int keep = p.k + (p.m > 0 ? p.m : 1);
   const int quota = (keep + TPR - 1) / TPR;
+  const int qstep = quota / 4 > 1 ? quota / 4 : 1;
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
   e = rr_once_per_device(attr_done, [] {
     cudaError_t a = cudaFuncSetAttribute(route_sweep_kernel<128>,
@@ -889,9 +867,9 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   const size_t smem = smem_bytes(p.d);
   if (p.d == 128)
-    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, force_hard);
+    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, qstep, force_hard);
   else
-    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, force_hard);
+    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, qstep, force_hard);
   rr_count_launch();
   return cudaPeekAtLastError();
 }

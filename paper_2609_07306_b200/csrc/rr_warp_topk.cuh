@@ -62,6 +62,67 @@ __device__ inline Sel warp_select(const uint32_t* keys, int v, int T, uint32_t* 
   return Sel{prefix, need, ties};
 }
 
+// Mandatory global sentinels and the random sentinel sample of one row (Section 3.1 items 2 and
+// 3, Section 3.4), by a whole warp.  bitmap: the row's excluded chunks (route + near-miss) as
+// ceil(v / 32) words in shared memory, private to the warp and updated here; pool = valid chunks
+// not excluded.  Sequential definition of the sample: pool <= r -> the whole pool in ascending
+// order; else for t = 0, 1, ...: j = floor(u_t v / 2^32), accepted iff j is not excluded and was
+// not drawn before, until r are accepted; after 64 r draws the smallest free chunks fill the
+// rest.  32 draws are examined per step: a draw is accepted iff its chunk is free in the bitmap
+// and no earlier lane of the step drew the same chunk; the accepted ones take the next slots in
+// lane (= draw) order, which is exactly the sequential outcome.
+__device__ __forceinline__ void sentinels_row(const RRParams& p, uint32_t* bitmap, int pool, int g,
+                                              int v, uint32_t layer, int lane) {
+  const unsigned lt = (1u << lane) - 1u;
+  int32_t* sent = p.sentinels + (size_t)g * p.sw;
+  if (p.n_global) {
+    int gi = 0;
+    for (int b = 0; b < 2; ++b) {
+      if (!((p.global_mask >> b) & 1)) continue;
+      const int j = b == 0 ? 0 : v - 1;
+      int id = -1;
+      if (v > 0) {
+        const uint32_t word = bitmap[j >> 5], bit = 1u << (j & 31);
+        if (!(word & bit)) { id = j; --pool; }
+        __syncwarp();
+        if (id >= 0 && lane == 0) bitmap[j >> 5] = word | bit;
+        __syncwarp();
+      }
+      if (lane == 0) sent[p.m + p.r + gi] = id;
+      ++gi;
+    }
+  }
+  int32_t* rnd = sent + p.m;
+  int taken = 0;
+  if (p.r > 0 && pool > 0) {
+    if (pool > p.r) {
+      const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
+      const int limit = 64 * p.r;
+      for (int t0 = 0; t0 < limit && taken < p.r; t0 += 32) {
+        const int j = (int)__umulhi(rr_draw_u32(rk, layer, (uint32_t)(t0 + lane)), (uint32_t)v);
+        const bool free_j = ((bitmap[j >> 5] >> (j & 31)) & 1u) == 0u;
+        const unsigned same = __match_any_sync(FULL, j);
+        const bool ok = t0 + lane < limit && free_j && (same & lt) == 0u;
+        const unsigned okmask = __ballot_sync(FULL, ok);
+        const int pos = taken + __popc(okmask & lt);
+        if (ok && pos < p.r) { rnd[pos] = j; atomicOr(&bitmap[j >> 5], 1u << (j & 31)); }
+        taken = min(p.r, taken + __popc(okmask));
+        __syncwarp();
+      }
+    }
+    // whole pool (pool <= r) or the bounded-work fill: smallest free chunks first
+    for (int j0 = 0; j0 < v && taken < p.r; j0 += 32) {
+      const int j = j0 + lane;
+      const bool fr = j < v && !((bitmap[j0 >> 5] >> lane) & 1u);
+      const unsigned bf = __ballot_sync(FULL, fr);
+      const int pos = taken + __popc(bf & lt);
+      if (fr && pos < p.r) rnd[pos] = j;
+      taken = min(p.r, taken + __popc(bf));
+    }
+  }
+  for (int s = taken + lane; s < p.r; s += 32) rnd[s] = -1;
+}
+
 // keys[0..v): the row's order keys (rr_order_key of the scores); hist: 256 words; bitmap:
 // ceil(n_k / 32) words.  All three in shared memory, private to the calling warp; bitmap and
 // hist need no initialisation.  g: global row id, v: chunks the row may select.
@@ -117,59 +178,8 @@ __device__ __forceinline__ void route_row(const RRParams& p, const uint32_t* key
   if (lane == 0) { p.kth[g] = kth; p.margin[g] = margin; }
   __syncwarp();
 
-  // random sentinels: r distinct chunks from the valid ones outside route and near-miss
-  // mandatory global sentinels (sink chunk, most recent chunk): a slot each after the random
-  // ones, empty if the chunk is already in the route or a near-miss sentinel
-  int pool = v - Tkeep;
-  if (p.n_global) {
-    int gi = 0;
-    for (int b = 0; b < 2; ++b) {
-      if (!((p.global_mask >> b) & 1)) continue;
-      const int j = b == 0 ? 0 : v - 1;
-      int id = -1;
-      if (v > 0) {
-        const uint32_t word = bitmap[j >> 5], bit = 1u << (j & 31);
-        if (!(word & bit)) { id = j; --pool; }
-        __syncwarp();
-        if (id >= 0 && lane == 0) bitmap[j >> 5] = word | bit;
-        __syncwarp();
-      }
-      if (lane == 0) sent[p.m + p.r + gi] = id;
-      ++gi;
-    }
-  }
-  int32_t* rnd = sent + p.m;
-  int taken = 0;
-  if (p.r > 0 && pool > 0) {
-    if (pool > p.r) {
-      const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
-      const int limit = 64 * p.r;
-      for (int t0 = 0; t0 < limit && taken < p.r; t0 += 32) {
-        const uint32_t u = rr_draw_u32(rk, layer, (uint32_t)(t0 + lane));
-        const int jmine = (int)__umulhi(u, (uint32_t)v);
-        for (int l = 0; l < 32 && taken < p.r && t0 + l < limit; ++l) {
-          const int jj = __shfl_sync(FULL, jmine, l);
-          const uint32_t word = bitmap[jj >> 5];
-          const uint32_t bit = 1u << (jj & 31);
-          if (!(word & bit)) {
-            if (lane == 0) { bitmap[jj >> 5] = word | bit; rnd[taken] = jj; }
-            ++taken;
-          }
-          __syncwarp();
-        }
-      }
-    }
-    // whole pool (pool <= r) or the bounded-work fill: smallest free chunks first
-    for (int j0 = 0; j0 < v && taken < p.r; j0 += 32) {
-      const int j = j0 + lane;
-      const bool fr = j < v && !((bitmap[j0 >> 5] >> lane) & 1u);
-      const unsigned bf = __ballot_sync(FULL, fr);
-      const int pos = taken + __popc(bf & lt);
-      if (fr && pos < p.r) rnd[pos] = j;
-      taken = min(p.r, taken + __popc(bf));
-    }
-  }
-  for (int s = taken + lane; s < p.r; s += 32) rnd[s] = -1;
+  __syncwarp();
+  sentinels_row(p, bitmap, v - Tkeep, g, v, layer, lane);
 }
 
 }  // namespace warptopk
