@@ -378,6 +378,23 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  int last = -1;
+  for (int t = BM - 1; t >= 0; --t) if (ctl->row[t] >= 0) { last = ctl->row[t]; break; }
+  const int vmax = rr_valid_count(last, p.n_k, p.causal, p.causal_offset);
+  const int n_tiles = (vmax + BN - 1) / BN;
+  const CUtensorMap* const tmap_ptr = &tmap_k;   // address in parameter space (what TMA needs)
+  // The Kc loads do not depend on the Qc tile: the ring's stages are filled (they are all free)
+  // and every Kc tile of the CTA is asked into L2 while the Qc rows are still on their way.
+  const int pre_q = min(H_STAGES, 2 * n_tiles * C::KHALVES);
+  if (tid == 0) {
+    for (int q = 0; q < pre_q; ++q) {
+      mbar_expect_tx(&ctl->full[q], C::B_HALF);
+      tma_load_3d(sB + q * C::B_HALF, tmap_ptr, (q % C::KHALVES) * 64, ((q / C::KHALVES) % n_tiles) * BN, prob, &ctl->full[q]);
+    }
+    for (int t = 0; t < n_tiles; ++t)
+#pragma unroll
+      for (int h = 0; h < C::KHALVES; ++h) tma_prefetch_l2_3d(tmap_ptr, h * 64, t * BN, prob);
+  }
   if (q_loader) {
     const uint32_t taddr = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_COL;
     if constexpr (QW == 64) tmem_st_32x64(taddr, qv); else tmem_st_32x32(taddr, qv);
@@ -389,24 +406,20 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   const uint32_t tmem_base = ctl->tmem_base;
   volatile uint32_t* abort_flag = &ctl->abort_flag;
 
-  int last = -1;
-  for (int t = BM - 1; t >= 0; --t) if (ctl->row[t] >= 0) { last = ctl->row[t]; break; }
-  const int vmax = rr_valid_count(last, p.n_k, p.causal, p.causal_offset);
-  const int n_tiles = (vmax + BN - 1) / BN;
-
   // Tiles are numbered through all sweeps (gt): stage and phase of every ring follow from gt.
   // producer / issuer: `first` .. `first + count` of that numbering
-  const CUtensorMap* const tmap_ptr = &tmap_k;   // address in parameter space (what TMA needs)
   // A stage of the Kc ring holds one K-half (64 of the d values) of a tile of 128 key chunks, so
   // that the load of a tile's first half can start as soon as the MMAs of the first half of the
   // tile two before it have finished.  Halves are numbered q = gt * KHALVES + h.
-  auto produce = [&](int first, int count) {
+  // (halves q < skip_q have been issued already)
+  auto produce = [&](int first, int count, int skip_q) {
     int issued = 0;
     for (int i = 0; i < count; ++i) {
       const int gt = first + i, t = gt % n_tiles;
 #pragma unroll
       for (int h = 0; h < C::KHALVES; ++h) {
         const int q = gt * C::KHALVES + h;
+        if (q < skip_q) { ++issued; continue; }
         const int s = q % H_STAGES; const uint32_t ph = (q / H_STAGES) & 1;
         if (!mbar_wait_spin(&ctl->empty[s], ph ^ 1, abort_flag)) { i = count; break; }
         mbar_expect_tx(&ctl->full[s], C::B_HALF);
@@ -511,12 +524,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 
   if (warp == 0) {
     if (lane == 0) {
-      // every Kc tile this CTA will walk is asked into L2 first: the tile loads of the sweeps
-      // then see L2 latency, not DRAM latency (two stages of shared memory hide little)
-      for (int t = 0; t < n_tiles; ++t)
-#pragma unroll
-        for (int h = 0; h < C::KHALVES; ++h) tma_prefetch_l2_3d(tmap_ptr, h * 64, t * BN, prob);
-      produce(0, 2 * n_tiles);
+      produce(0, 2 * n_tiles, pre_q);
     }
     __syncwarp();
   } else if (!is_sel) {
@@ -765,7 +773,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     // decision to stop after a timed-out wait the same for every thread
     if (__syncthreads_or((int)ctl->abort_flag)) break;
     if (warp == 0) {
-      if (lane == 0) produce(next_gt, n_tiles);
+      if (lane == 0) produce(next_gt, n_tiles, 0);
       __syncwarp();
     } else if (!is_sel) {
       if (lane == 0) issue(next_gt, n_tiles, warp == 1 ? 0 : 1);
