@@ -278,7 +278,8 @@ def run_ours(args) -> None:
     if w.dtype == W.DTYPE_BF16:
         dq, dk = dq.view(torch.bfloat16), dk.view(torch.bfloat16)
 
-    cfg = config_from_workload(w, two_pass=args.two_pass, gathered=args.gathered)
+    cfg = config_from_workload(w, two_pass=args.two_pass, gathered=args.gathered,
+                               streaming=args.streaming, inplace=args.inplace)
     led = RouteLedger(cfg, device=str(dev))
     stream = torch.cuda.current_stream(dev)
 
@@ -511,6 +512,11 @@ def main():
                     help="warm-up + timed steps only (for profiler captures)")
     ap.add_argument("--two-pass", action="store_true",
                     help="route through score rows in scratch + warp-level TopK")
+    ap.add_argument("--streaming", action="store_true",
+                    help="route with the streaming fused kernel instead of the two-sweep kernel")
+    ap.add_argument("--inplace", action="store_true",
+                    help="relay layers: challenge test inside the routing kernel (one pass over "
+                         "the score strip, no compacted second GEMM)")
     ap.add_argument("--gathered", action="store_true",
                     help="rescore candidates with the gathered FP32 kernel")
     args = ap.parse_args()

@@ -83,7 +83,11 @@ typedef struct rr_config {
                               bit 3 (tests): the two-sweep routing kernel hands every fifth
                               row to its exact slow path;
                               bit 4: route with the streaming fused kernel even where the
-                              two-sweep kernel applies                                     */
+                              two-sweep kernel applies;
+                              bit 5: relay in place -- the challenge test of Eq. 5 runs inside
+                              the routing kernel on the scores of its first sweep (no separate
+                              rescoring kernel, no second score GEMM over a compacted list);
+                              the results are the same                                     */
   /* Optional policies either side of the trigger; all zero = the plain method.             */
   int32_t global_sentinels;/* mandatory global candidates (Section 3.1, item 3): bit 0 = the
                               sink chunk 0, bit 1 = the most recent chunk the row may select.

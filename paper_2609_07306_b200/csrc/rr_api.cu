@@ -149,7 +149,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     // Section 4.1: the anchor builds the state from a complete chunk-score matrix.
     LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, L->dense_pairs_per_layer, st));
     if (L->sweep) {
-      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer,
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer, 0,
                                                         (L->cfg.debug_outputs >> 3) & 1, st));
       LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, nullptr, layer, st));
     } else if (L->fused) {
@@ -162,12 +162,23 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     L->anchored = 1;
   } else {
     if (!L->anchored) return RR_ERR_STATE;
+    if (L->inplace) {
+      // Relay in one pass over the score strip: the routing kernel tests every row (Eq. 5) on
+      // the scores of its first sweep and re-routes the failing rows in place; the compaction
+      // kernel then only builds the list the caller sees (and the sentinel kernel works from).
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer, 1,
+                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+      LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
+      LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, p.refresh_rows, layer, st));
+      if (p.chunk_tokens > 0) LAUNCH(RR_KIND_EXPAND, rr_launch_expand(p, 0, st));
+      return RR_OK;
+    }
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
     if (L->dense_rescore) LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, st));
     else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
     if (L->sweep) {
-      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, p.refresh_rows, layer,
+      LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, p.refresh_rows, layer, 0,
                                                         (L->cfg.debug_outputs >> 3) & 1, st));
       LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, p.refresh_rows, layer, st));
     } else if (L->fused) {
@@ -251,6 +262,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
   L->sweep = uses_sweep(cfg);
+  L->inplace = L->sweep && (cfg->debug_outputs & 32) && rr_route_sweep_inplace_supported(p);
   L->fused = uses_fused(cfg);
   L->dense_rescore = !(cfg->debug_outputs & 4) && rr_rescore_dense_supported(p);
   *out = L;

@@ -40,6 +40,7 @@ struct rr_ledger {
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
   bool sweep;                              // full routing runs in the two-sweep fused kernel
+  bool inplace;                            // relay: challenge test inside the routing kernel
   bool fused;                              // ... else in the streaming fused kernel
   bool dense_rescore;                      // relay rescoring reads the tensor-core score strip
   unsigned long long dense_pairs_per_layer;
@@ -113,8 +114,9 @@ cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void*
                                   const int32_t* row_list, int layer, cudaStream_t st);
 bool rr_route_sweep_supported(const RRParams& p);
 cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void* kc,
-                                  const int32_t* row_list, int layer, int force_hard,
+                                  const int32_t* row_list, int layer, int inplace, int force_hard,
                                   cudaStream_t st);
+bool rr_route_sweep_inplace_supported(const RRParams& p);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
 // global + random sentinels of the listed rows (after rr_launch_route_sweep; n_k <= 1024)

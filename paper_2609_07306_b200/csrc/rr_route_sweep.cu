@@ -51,6 +51,7 @@ constexpr int CAPJ = 32;                           // entries per list
 constexpr int MAX_KEEP = 48, MAX_NK = 1024;        // what the lists / bitmaps are sized for
 constexpr int BM_WORDS = MAX_NK / 32;
 constexpr int HARD_SLOTS = 24;                     // score rows held at once by the slow path
+constexpr int MAX_SLOTS = 16;                      // candidate slots per thread of the in-place relay
 constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr uint32_t ENTRY_PITCH = TPR * BM * 8;     // bytes between entries e and e+1 of a list
 constexpr uint32_t LIST_PITCH = BM * 8;            // bytes between lists j and j+1 of a row
@@ -66,13 +67,17 @@ struct Ctl {
   uint32_t tmem_base, abort_flag, hard_n, pad_;
   int row[BM], slot[BM];
   float tau_row[BM];                // the row's bound from the group maxima
+  float ab[2][TPR][BM];             // in-place relay: each thread's part of alpha / beta
+  uint32_t n_flagged, n_cand, pad2_[2];
+  unsigned long long v_flagged;     // in-place relay: counters of the CTA
+  uint8_t live[BM];                 // in-place relay: the row failed the challenge test
   uint32_t cnt[TPR][BM];            // list lengths; bit 8 = this list needs the slow path
   uint32_t cut_k[BM], cut_keep[BM]; // per row: entries of each list (8 bits each) in the top k / keep
   uint8_t cut_bad[2][BM];           // a cut could not be settled (scores tie across it)
   uint8_t hard_rows[BM];            // rows handed to the slow path, in registration order
   int8_t hard_slot[BM];             // position of a row in hard_rows, -1 = none
 };
-constexpr int CTL_BYTES = 8192;
+constexpr int CTL_BYTES = 12288;
 static_assert(sizeof(Ctl) <= CTL_BYTES, "control block too large");
 constexpr int BUF_BYTES = CAPJ * ENTRY_PITCH;             // 128 KB
 static_assert(HARD_SLOTS * MAX_NK * 4 + SEL_WARPS * (256 + BM_WORDS) * 4 <= BUF_BYTES,
@@ -306,7 +311,7 @@ template <int D>
 __global__ void __launch_bounds__(NT, 1)
 route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
-                   uint32_t layer, int quota, int qstep, int force_hard) {
+                   uint32_t layer, int inplace, int force_hard) {
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -371,6 +376,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     }
     ctl->abort_flag = 0;
     ctl->hard_n = 0;
+    ctl->n_flagged = 0; ctl->n_cand = 0; ctl->v_flagged = 0ull;
     mbar_fence_init();
     tma_prefetch_desc(&tmap_k);
   }
@@ -536,6 +542,28 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     if (lane == 0) PH_CNT(7, ph_t0_ - cta_t0_);
 #endif
     // ===== sweep 1: group maxima -> tau ==========================================================
+    // In-place relay (Section 3.2 on the same score strip): every thread also dumps its scores of
+    // the tile to shared memory ([column][row], two tiles in the still unused list area), and after
+    // a barrier of the row's four threads looks up the current scores of its share of the row's
+    // candidates: alpha = min over route slots, beta = max over sentinel slots (Eq. 5).
+    int cid[MAX_SLOTS];
+    const int slots = (p.c + TPR - 1) / TPR, slot0 = jslice * slots;
+    float a_part = pinf, b_part = ninf;
+    int n_cand = 0; bool bad_id = false;
+    if (inplace) {
+#pragma unroll
+      for (int q = 0; q < MAX_SLOTS; ++q) {
+        const int sl = slot0 + q;
+        int id = -1;
+        if (row >= 0 && q < slots && sl < p.c)
+          id = sl < p.k ? p.routes[(size_t)g * p.k + sl] : p.sentinels[(size_t)g * p.sw + (sl - p.k)];
+        bad_id |= id >= v;
+        cid[q] = id >= 0 && id < v ? id : -1;
+        n_cand += cid[q] >= 0;
+        if (p.debug && row >= 0 && q < slots && sl < p.c)
+          p.cand_scores[(size_t)g * p.c + sl] = __int_as_float(0x7fc00000);
+      }
+    }
     float mx[SLICE];
 #pragma unroll
     for (int i = 0; i < SLICE; ++i) mx[i] = ninf;
@@ -552,27 +580,38 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
           for (int i = 0; i < SLICE; ++i)
             mx[i] = col0 + i < v ? fmaxf(mx[i], __uint_as_float(acc[i])) : mx[i];
         }
+        if (inplace) {
+          const uint32_t dump = buf0 + (uint32_t)(t & 1) * (BN * BM * 4u) + (uint32_t)(jslice * SLICE) * (BM * 4u) + (uint32_t)r * 4u;
+#pragma unroll
+          for (int i = 0; i < SLICE; ++i) sts32(dump + (uint32_t)i * (BM * 4u), acc[i]);
+        }
       }
       tile_release(t);
+      if (inplace) {
+        quarter_sync(quarter);
+        const uint32_t tile_dump = buf0 + (uint32_t)(t & 1) * (BN * BM * 4u) + (uint32_t)r * 4u;
+#pragma unroll
+        for (int q = 0; q < MAX_SLOTS; ++q) {
+          const int id = cid[q];
+          if (id >= 0 && (id >> 7) == t) {
+            const float sc = __uint_as_float(lds32(tile_dump + (uint32_t)(id & (BN - 1)) * (BM * 4u)));
+            if (slot0 + q < p.k) a_part = fminf(a_part, sc); else b_part = fmaxf(b_part, sc);
+            if (p.debug) p.cand_scores[(size_t)g * p.c + slot0 + q] = sc;
+          }
+        }
+      }
+    }
+    if (inplace) {
+      ctl->ab[0][jslice][r] = a_part; ctl->ab[1][jslice][r] = b_part;
+      if (__any_sync(FULL, bad_id) && lane == 0) atomicOr(p.status, RR_STATUS_BAD_INDEX);
+      n_cand = __reduce_add_sync(FULL, n_cand);
+      if (lane == 0) atomicAdd(&ctl->n_cand, (uint32_t)n_cand);
+      // every selection warp of the CTA has read its last dump: the list area (which the dumps of
+      // all quarters share) is free
+      asm volatile("bar.sync 5, %0;" ::"n"(SEL_WARPS * 32) : "memory");
     }
     PH_LAP(0);
-#ifdef RR_LOCKSTEP
-    asm volatile("bar.sync 5, 512;" ::: "memory");
-    PH_LAP(14);
-#endif
     OESort<0, SLICE, float, DescF<float>, SLICE>::run(mx);
-#ifdef RR_ICACHE_PROBE
-    PH_LAP(11);
-    // the same code again on a copy (a value the compiler cannot know keeps it from folding)
-    for (int rep_ = 0; rep_ < 2; ++rep_) {
-      float my[SLICE];
-#pragma unroll
-      for (int i = 0; i < SLICE; ++i) my[i] = mx[(i * 7) & 31] + (float)(quota >> 20);
-      OESort<0, SLICE, float, DescF<float>, SLICE>::run(my);
-      if (my[0] < my[31]) mx[0] = my[5];
-      if (rep_ == 0) PH_LAP(12); else PH_LAP(13);
-    }
-#endif
     // The row's keep-th largest group maximum (over the 128 groups of its four threads) has keep
     // distinct scores of the row at or above it: a valid inclusive lower bound of the row's
     // keep-th largest score, and the tightest one the maxima give (about 1.2 keep scores pass;
@@ -594,6 +633,21 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                                           q_ + (1 < rm_), q_ + (2 < rm_), q_, bounded, MAX_KEEP);
       if (bounded) tau = ex.lo;
       ctl->tau_row[r] = tau;
+      if (inplace) {
+        // challenge test of the row (Eq. 5 and the optional policies): only rows that fail it are
+        // routed again; the others keep their ledger row
+        const float alpha = fminf(fminf(ctl->ab[0][0][r], ctl->ab[0][1][r]), fminf(ctl->ab[0][2][r], ctl->ab[0][3][r]));
+        const float beta = fmaxf(fmaxf(ctl->ab[1][0][r], ctl->ab[1][1][r]), fmaxf(ctl->ab[1][2][r], ctl->ab[1][3][r]));
+        const bool flag = row >= 0 && rr_challenge(p, g, alpha, beta);
+        ctl->live[r] = flag;
+        if (row >= 0) { p.flags[g] = flag ? 1 : 0; p.alpha[g] = alpha; p.beta[g] = beta; }
+        const int n_flag = __popc(__ballot_sync(FULL, flag));
+        const int v_sum = __reduce_add_sync(FULL, flag ? v : 0);
+        if (lane == 0) {
+          atomicAdd(&ctl->n_flagged, (uint32_t)n_flag);
+          atomicAdd(&ctl->v_flagged, (unsigned long long)v_sum);
+        }
+      }
     }
     PH_LAP(10);
     quarter_sync(quarter);                  // the published maxima have been read: lists are free
@@ -601,7 +655,8 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     // rows of a refresh list also have the bound the rescoring kernel derived from the old
     // candidates' current scores (bit-identical scores: no margin needed)
     if (row_list && row >= 0) tau = fmaxf(tau, p.tau[g]);
-    if (row < 0) tau = pinf;                               // padding rows pass nothing
+    const bool routed = row >= 0 && (!inplace || ctl->live[r] != 0);   // this row is (re)routed here
+    if (!routed) tau = pinf;                               // padding / reused rows pass nothing
     PH_LAP(1);
 
     // ===== sweep 2: threshold filter into this thread's list ====================================
@@ -626,10 +681,6 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     const int n = min(n_raw, CAPJ);
 
     // ===== sort the list (network sized for the longest list of the warp) =========================
-#ifdef RR_LOCKSTEP
-    asm volatile("bar.sync 5, 512;" ::: "memory");
-    PH_LAP(15);
-#endif
     {
       const int n_warp = __reduce_max_sync(FULL, n);
       bool run3;
@@ -643,7 +694,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     if (row >= 0 && slow && n_raw <= CAPJ) PH_CNT(18, 1);
     if (row >= 0) { PH_CNT(22, n_raw); PH_CNT(23, 1); }
 #endif
-    if (force_hard && row >= 0 && g % 5 == 0) slow = true;     // test hook: exercise the slow path
+    if (force_hard && routed && g % 5 == 0) slow = true;     // test hook: exercise the slow path
     ctl->cnt[jslice][r] = (uint32_t)n | (slow ? 256u : 0u);
     PH_LAP(3);
     quarter_sync(quarter);
@@ -656,7 +707,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     // every other one <= hi; lo > hi settles the set exactly, lo == hi (equal scores across the
     // cut) is left to the slow path.  The k cut also yields the k-th score (lo) and the margin.
     const uint32_t c0 = ctl->cnt[0][r], c1 = ctl->cnt[1][r], c2 = ctl->cnt[2][r], c3 = ctl->cnt[3][r];
-    const bool have = alive && row >= 0;
+    const bool have = alive && routed;
     const bool hard_list = have && ((c0 | c1 | c2 | c3) & 256u) != 0u;
     const bool go0 = have && !hard_list;
     const int n_total = (int)((c0 & 255u) + (c1 & 255u) + (c2 & 255u) + (c3 & 255u));
@@ -821,6 +872,12 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
     if (lane == 0 && ctl->abort_flag) atomicOr(p.status, RR_STATUS_TIMEOUT);
+    if (lane == 0 && inplace) {      // what the compaction kernel and the work counters need
+      p.tile_counts[prob * tiles_m + tm] = (int)ctl->n_flagged;
+      atomicAdd(&p.counters[RR_CNT_FLAGGED_ROWS], (unsigned long long)ctl->n_flagged);
+      atomicAdd(&p.counters[RR_CNT_CAND_PAIRS], (unsigned long long)ctl->n_cand);
+      atomicAdd(&p.counters[RR_CNT_FULL_PAIRS], ctl->v_flagged);
+    }
   }
 }
 
@@ -852,17 +909,20 @@ bool rr_route_sweep_supported(const RRParams& p) {
          smem_bytes(p.d) <= 227 * 1024;
 }
 
+// The in-place relay holds a row's candidates in 16 registers of each of its four threads.
+bool rr_route_sweep_inplace_supported(const RRParams& p) {
+  return rr_route_sweep_supported(p) && p.c <= TPR * MAX_SLOTS;
+}
+
 cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void* kc,
-                                  const int32_t* row_list, int layer, int force_hard,
+                                  const int32_t* row_list, int layer, int inplace, int force_hard,
                                   cudaStream_t st) {
+  if (inplace && (row_list || p.c > TPR * MAX_SLOTS)) return cudaErrorInvalidConfiguration;
   if (!rr_route_sweep_supported(p)) return cudaErrorInvalidConfiguration;
   CUtensorMap tmap;
   cudaError_t e = rr_encode_tmap_bf16_3d(&tmap, kc, p.d, p.n_k, p.P, BN);
   if (e != cudaSuccess) return e;
   const int grid = p.P * p.tiles_per_problem;
-  const int keep = p.k + (p.m > 0 ? p.m : 1);
-  const int quota = (keep + TPR - 1) / TPR;
-  const int qstep = quota / 4 > 1 ? quota / 4 : 1;
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
   e = rr_once_per_device(attr_done, [] {
     cudaError_t a = cudaFuncSetAttribute(route_sweep_kernel<128>,
@@ -875,9 +935,9 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   const size_t smem = smem_bytes(p.d);
   if (p.d == 128)
-    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, qstep, force_hard);
+    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, force_hard);
   else
-    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, quota, qstep, force_hard);
+    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, force_hard);
   rr_count_launch();
   return cudaPeekAtLastError();
 }

@@ -79,7 +79,8 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
                        layers: Optional[int] = None, gen_threads: int = 8,
                        report: Optional[ParityReport] = None,
                        two_pass: bool = False, gathered: bool = False,
-                       force_slow_rows: bool = False, streaming: bool = False) -> ParityReport:
+                       force_slow_rows: bool = False, streaming: bool = False,
+                       inplace: bool = False) -> ParityReport:
     """Runs `layers` layers of workload w on the device over ALL problems and checks the
     listed problems (default all) against the oracle with teacher forcing."""
     rep = report or ParityReport()
@@ -90,7 +91,7 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
     q_all, k_all = W.generate(w, problems=all_problems, layers=L, threads=gen_threads)
     led = RouteLedger(config_from_workload(w, debug_outputs=True, two_pass=two_pass,
                                            gathered=gathered, force_slow_rows=force_slow_rows,
-                                           streaming=streaming))
+                                           streaming=streaming, inplace=inplace))
     rows_sel = np.concatenate([np.arange(pr * w.n_q, (pr + 1) * w.n_q) for pr in check])
     sel_t = torch.from_numpy(rows_sel).cuda()
     v_sel = np.tile(p.valid_counts(), len(check))

@@ -45,18 +45,19 @@ def test_sweep_shapes(n, two_pass, gathered):
     parity.assert_clean(rep)
 
 
-@pytest.mark.parametrize("variant", ["slow_rows", "streaming"])
+@pytest.mark.parametrize("variant", ["slow_rows", "streaming", "inplace", "inplace+slow_rows"])
 @pytest.mark.parametrize("wl", ["moderate", "sweep512", "sweep1024"])
 def test_routing_kernel_variants(wl, variant):
-    """The two other ways a bf16 row can be routed in one kernel: the two-sweep kernel with every
+    """The other ways a bf16 row can be routed in one kernel (and "inplace": the relay whose
+    challenge test runs inside the routing kernel, Section 3.2 and 4.2 in one pass): the two-sweep kernel with every
     fifth row handed to its exact slow path (complete score row in shared memory + warp-level
     radix select), and the streaming kernel that serves the shapes the two-sweep kernel does
     not hold."""
     w = {"moderate": W.moderate(),
          "sweep512": W.sweep(512, 0.15).replace(heads=4, layers=4, anchor_every=3),
          "sweep1024": W.sweep(1024, 0.30).replace(heads=3, layers=3, anchor_every=2)}[wl]
-    rep = parity.run_teacher_forced(w, force_slow_rows=variant == "slow_rows",
-                                    streaming=variant == "streaming")
+    rep = parity.run_teacher_forced(w, force_slow_rows="slow_rows" in variant,
+                                    streaming=variant == "streaming", inplace="inplace" in variant)
     _report(rep)
     parity.assert_clean(rep)
 
