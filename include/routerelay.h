@@ -58,7 +58,6 @@ extern "C" {
 /* bits of the device status word (rr_ledger_status) */
 #define RR_STATUS_TIMEOUT      1u  /* an mbarrier wait in a kernel gave up                     */
 #define RR_STATUS_BAD_INDEX    2u  /* a ledger entry outside [0, v_i) was met and skipped      */
-#define RR_STATUS_OVERFLOW     4u  /* an internal per-row buffer overflowed (result invalid)   */
 
 typedef struct rr_ledger rr_ledger;   /* opaque; owns only a small host struct */
 
@@ -87,7 +86,11 @@ typedef struct rr_config {
                               bit 5: relay in place -- the challenge test of Eq. 5 runs inside
                               the routing kernel on the scores of its first sweep (no separate
                               rescoring kernel, no second score GEMM over a compacted list);
-                              the results are the same                                     */
+                              the results are the same;
+                              bits 6, 7 (tests): the first wait of the first CTA of the first
+                              routing launch (bit 6) / strip rescoring launch (bit 7) of this
+                              ledger counts as expired, once: that CTA gives up as after a real
+                              time-out and the status word gets RR_STATUS_TIMEOUT          */
   /* Optional policies either side of the trigger; all zero = the plain method.             */
   int32_t global_sentinels;/* mandatory global candidates (Section 3.1, item 3): bit 0 = the
                               sink chunk 0, bit 1 = the most recent chunk the row may select.
@@ -206,7 +209,10 @@ int rr_ledger_export(rr_ledger* L, void* host_blob, size_t bytes, void* stream);
 int rr_ledger_import(rr_ledger* L, const void* host_blob, size_t bytes, void* stream);
 
 /* Synchronous read of the device status word (RR_STATUS_* bits); RR_ERR_TIMEOUT is
- * returned if the timeout bit is set. */
+ * returned if the timeout bit is set.  A CTA whose bounded wait expired leaves its rows as
+ * they were (a relay may then hold flags and a refresh list that disagree for those rows; all
+ * writes stay in bounds): after RR_ERR_TIMEOUT the ledger's contents are not to be used --
+ * rr_ledger_reset (which clears the status word) and a new anchor bring it back. */
 int rr_ledger_status(rr_ledger* L, void* stream, uint32_t* status_out);
 
 /* Host-callable copy of the sampler's counter-based generator (the t-th 32-bit draw of

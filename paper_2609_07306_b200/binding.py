@@ -25,7 +25,6 @@ RR_BF16 = 0
 RR_F32 = 1
 RR_STATUS_TIMEOUT = 1
 RR_STATUS_BAD_INDEX = 2
-RR_STATUS_OVERFLOW = 4
 RR_NUM_COUNTERS = 8
 RR_NUM_KINDS = 12
 COUNTER_NAMES = ("layer_calls", "anchor_rows", "relay_rows", "flagged_rows", "cand_pairs",

@@ -129,6 +129,13 @@ unsigned long long dense_pairs(const rr_config* c) {
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
+// test hooks of the next routing launch: slow rows (debug bit 3), one forced time-out (bit 6)
+int sweep_hooks(rr_ledger* L) {
+  int h = (L->cfg.debug_outputs >> 3) & 1;
+  if (L->timeout_shots & 1) { h |= 2; L->timeout_shots &= ~1; }
+  return h;
+}
+
 int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool anchor,
                 cudaStream_t st) {
   if (!L || !qc || !kc || layer < 0) return RR_ERR_INVALID_ARG;
@@ -150,7 +157,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     LAUNCH(RR_KIND_ANCHOR_FILL, rr_launch_anchor_fill(p, L->dense_pairs_per_layer, st));
     if (L->sweep) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer, 0,
-                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+                                                        sweep_hooks(L), st));
       LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, nullptr, layer, st));
     } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, nullptr, layer, st));
@@ -167,19 +174,23 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
       // the scores of its first sweep and re-routes the failing rows in place; the compaction
       // kernel then only builds the list the caller sees (and the sentinel kernel works from).
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, nullptr, layer, 1,
-                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+                                                        sweep_hooks(L), st));
       LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
       LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, p.refresh_rows, layer, st));
       if (p.chunk_tokens > 0) LAUNCH(RR_KIND_EXPAND, rr_launch_expand(p, 0, st));
       return RR_OK;
     }
     // Section 4.2: rescoring + flags, prefix-sum compaction, refresh of the listed rows.
-    if (L->dense_rescore) LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, st));
+    if (L->dense_rescore) {
+      const int shot = (L->timeout_shots >> 1) & 1;     // test hook: one forced time-out
+      L->timeout_shots &= ~2;
+      LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, shot, st));
+    }
     else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));
     if (L->sweep) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_sweep(p, qc, kc, p.refresh_rows, layer, 0,
-                                                        (L->cfg.debug_outputs >> 3) & 1, st));
+                                                        sweep_hooks(L), st));
       LAUNCH(RR_KIND_SENTINELS, rr_launch_sentinels(p, p.refresh_rows, layer, st));
     } else if (L->fused) {
       LAUNCH(RR_KIND_ROUTE_FUSED, rr_launch_route_fused(p, qc, kc, p.refresh_rows, layer, st));
@@ -240,6 +251,7 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   L->dev_scratch = dev_scratch; L->scratch_bytes = scratch_bytes;
   L->export_bytes = lay.export_total;
   L->anchored = 0;
+  L->timeout_shots = (cfg->debug_outputs >> 6) & 3;
   L->device = -1;
   cudaGetDevice(&L->device);           // informational; failure (no GPU) leaves -1
   cudaGetLastError();

@@ -39,6 +39,8 @@ struct rr_ledger {
   size_t export_bytes;
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
+  int timeout_shots;                       // test hook: forced time-outs still to be fired (bit 0
+                                           // routing kernel, bit 1 strip rescoring kernel)
   bool sweep;                              // full routing runs in the two-sweep fused kernel
   bool inplace;                            // relay: challenge test inside the routing kernel
   bool fused;                              // ... else in the streaming fused kernel
@@ -114,8 +116,8 @@ cudaError_t rr_launch_route_fused(const RRParams& p, const void* qc, const void*
                                   const int32_t* row_list, int layer, cudaStream_t st);
 bool rr_route_sweep_supported(const RRParams& p);
 cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void* kc,
-                                  const int32_t* row_list, int layer, int inplace, int force_hard,
-                                  cudaStream_t st);
+                                  const int32_t* row_list, int layer, int inplace, int hooks,
+                                  cudaStream_t st);   // hooks: bit 0 slow rows, bit 1 forced time-out
 bool rr_route_sweep_inplace_supported(const RRParams& p);
 cudaError_t rr_launch_topk_rows(const RRParams& p, const int32_t* row_list, int layer,
                                 cudaStream_t st);
@@ -126,7 +128,7 @@ cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
                               cudaStream_t st);
 bool rr_rescore_dense_supported(const RRParams& p);
 cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
-                                    cudaStream_t st);
+                                    int force_timeout, cudaStream_t st);
 // compact / anchor_fill also advance the ages and the cumulative counters of the layer
 cudaError_t rr_launch_compact(const RRParams& p, unsigned long long dense_pairs, cudaStream_t st);
 cudaError_t rr_launch_anchor_fill(const RRParams& p, unsigned long long dense_pairs,

@@ -72,7 +72,7 @@ __device__ unsigned long long g_rd_phase[8];
 template <int D>
 __global__ void __launch_bounds__(NT, 2)
 rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
-                     const __grid_constant__ CUtensorMap tmap_k, int words) {
+                     const __grid_constant__ CUtensorMap tmap_k, int words, int force_timeout) {
   using P = tcpipe::Pipe<D, BN, B_STAGES, ACC_STAGES, NCONS>;
   extern __shared__ uint8_t smem_raw[];
   P pipe;
@@ -206,6 +206,8 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
     RD_LAP(1);
     for (int t = 0; t < n_tiles; ++t) {
       // after a wait that gave up the remaining iterations only keep the barriers in step
+      // (test hook: the first wait of CTA 0 counts as expired)
+      if (force_timeout && blockIdx.x == 0 && t == 0) { pipe.ctl->abort_flag = 1u; alive = false; }
       if (alive) alive = pipe.consumer_wait(t);
       RD_LAP(2);
       static_assert(COLS == 32, "a thread's share of a tile is one bitmap word");
@@ -311,7 +313,7 @@ bool rr_rescore_dense_supported(const RRParams& p) {
 }
 
 cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
-                                    cudaStream_t st) {
+                                    int force_timeout, cudaStream_t st) {
   int words;
   const size_t smem = smem_need(p, words);
   CUtensorMap tmap, tmap_q;
@@ -334,9 +336,9 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
   if (e != cudaSuccess) return e;
   const int grid = p.n_tiles;
   if (p.d == 128)
-    rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words);
+    rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
   else
-    rescore_dense_kernel<64><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words);
+    rescore_dense_kernel<64><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
   rr_count_launch();
   return cudaPeekAtLastError();
 }

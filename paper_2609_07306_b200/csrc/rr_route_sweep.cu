@@ -64,6 +64,7 @@ struct Cfg {
 
 struct Ctl {
   uint64_t full[H_STAGES], empty[H_STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+  uint64_t drain[ISSUE_WARPS];       // completes when all MMAs of an issuer have finished
   uint32_t tmem_base, abort_flag, hard_n, pad_;
   int row[BM], slot[BM];
   float tau_row[BM];                // the row's bound from the group maxima
@@ -311,7 +312,8 @@ template <int D>
 __global__ void __launch_bounds__(NT, 1)
 route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
-                   uint32_t layer, int inplace, int force_hard) {
+                   uint32_t layer, int inplace, int hooks) {
+  const bool force_hard = hooks & 1, force_timeout = hooks & 2;      // test hooks
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -374,6 +376,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
       mbar_init(&ctl->acc_full[s], 1);
       mbar_init(&ctl->acc_empty[s], SEL_WARPS);          // one arrival per selection warp
     }
+    for (int s = 0; s < ISSUE_WARPS; ++s) mbar_init(&ctl->drain[s], 1);
     ctl->abort_flag = 0;
     ctl->hard_n = 0;
     ctl->n_flagged = 0; ctl->n_cand = 0; ctl->v_flagged = 0ull;
@@ -511,6 +514,9 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   auto tile_wait = [&](int gt) -> int {
     const int as = gt % ACC_STAGES; const uint32_t aph = (gt / ACC_STAGES) & 1;
     if (alive) {
+      // test hook: the first wait of CTA 0 counts as expired (what a wait that ran out does:
+      // raise the CTA's abort flag; every role then leaves its loop at its next poll)
+      if (force_timeout && blockIdx.x == 0 && gt == 0) *abort_flag = 1u;
       const bool ready = mbar_wait_warp(&ctl->acc_full[as], aph, abort_flag, 20);
       if (!__all_sync(FULL, ready)) alive = false;
     }
@@ -863,6 +869,13 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     }
   }
 
+  // TMEM must not be freed while an MMA can still write to it: after a wait that gave up the
+  // consumers no longer vouch for that, so each issuer waits (bounded) for its own MMAs
+  if (!is_sel && warp != 0 && lane == 0) {
+    const int which = warp == 1 ? 0 : 1;
+    umma_commit(&ctl->drain[which]);
+    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->drain[which], 0); ++it) __nanosleep(64);
+  }
   tc_fence_before();
   __syncthreads();
 #ifdef RR_PHASE_TIMING
@@ -915,7 +928,7 @@ bool rr_route_sweep_inplace_supported(const RRParams& p) {
 }
 
 cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void* kc,
-                                  const int32_t* row_list, int layer, int inplace, int force_hard,
+                                  const int32_t* row_list, int layer, int inplace, int hooks,
                                   cudaStream_t st) {
   if (inplace && (row_list || p.c > TPR * MAX_SLOTS)) return cudaErrorInvalidConfiguration;
   if (!rr_route_sweep_supported(p)) return cudaErrorInvalidConfiguration;
@@ -935,9 +948,9 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   const size_t smem = smem_bytes(p.d);
   if (p.d == 128)
-    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, force_hard);
+    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks);
   else
-    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, force_hard);
+    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks);
   rr_count_launch();
   return cudaPeekAtLastError();
 }

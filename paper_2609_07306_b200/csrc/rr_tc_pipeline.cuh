@@ -34,6 +34,7 @@ struct Pipe {
   struct Ctl {
     uint64_t full[B_STAGES], empty[B_STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
     uint64_t a_full;                                      // Qc tile landed (TMA variant only)
+    uint64_t drain;                                       // all MMAs of the issuer have finished
     uint32_t tmem_base, abort_flag;
     int row[BM], slot[BM];
   };
@@ -71,6 +72,7 @@ struct Pipe {
       for (int s = 0; s < B_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
       for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(&ctl->acc_full[s], 1); mbar_init(&ctl->acc_empty[s], CONSUMERS); }
       mbar_init(&ctl->a_full, 1);
+      mbar_init(&ctl->drain, 1);
       ctl->abort_flag = 0;
       mbar_fence_init();
       tma_prefetch_desc(tmap_k);
@@ -158,6 +160,10 @@ struct Pipe {
       umma_commit(&ctl->empty[s]);        // smem stage reusable once these MMAs have read it
       umma_commit(&ctl->acc_full[as]);    // accumulator ready for the consumers
     }
+    // TMEM must not be freed while an MMA can still write to it: after a wait that gave up the
+    // consumers no longer vouch for that, so the issuer waits (bounded) for its own MMAs
+    umma_commit(&ctl->drain);
+    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->drain, 0); ++it) __nanosleep(64);
   }
 
   // Consumer side of one tile: returns false (for the whole warp) if the wait gave up.
