@@ -74,6 +74,27 @@ def _oracle_sample(w: W.RouteWorkload, n_problems: int, n_layers: int):
                                 f"{w.layers} layers ({rows} row-layers, {dt:.1f} s)"
 
 
+def _timed_sample(w: W.RouteWorkload, n_problems: int, n_layers: int, repeats: int = 5):
+    """Times the oracle's vectorised fp32 mode (BLAS matmul + argpartition) on a sample of the
+    workload; median of `repeats` runs."""
+    from oracle import routerelay_timed as T
+    problems = list(range(min(n_problems, w.problems)))
+    n_layers = min(n_layers, w.layers)
+    q, k = W.generate(w, problems=problems, layers=n_layers)
+    qf, kf = W.as_float32(q), W.as_float32(k)
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        T.run_layers(qf, kf, w.n_q, w.n_k, w.k, w.m, w.r, w.gamma, w.causal, w.seed,
+                     w.anchor_every, problems)
+        times.append(time.perf_counter() - t0)
+    dt = statistics.median(times)
+    rows = len(problems) * w.n_q * n_layers
+    return rows / dt, dt, f"{len(problems)} of {w.problems} problems x first {n_layers} of " \
+                          f"{w.layers} layers ({rows} row-layers, median of {repeats} runs, " \
+                          f"{dt:.2f} s each)"
+
+
 def _blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -93,16 +114,16 @@ def run_reference(args) -> None:
         v, dt, summ, sample = _oracle_sample(w, 2, 5)
         if s >= args.warmup:
             vals.append((v, dt))
-    value = sum(v for v, _ in vals) / len(vals)
-    ms = 1e3 * sum(dt for _, dt in vals) / len(vals)
+    ms = 1e3 * statistics.median(dt for _, dt in vals)
+    value = statistics.median(v for v, _ in vals)
     cores = _blas_threads()
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "sample_per_step": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores,
+                         "os_cpu_count": os.cpu_count(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -199,6 +220,10 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
             out["hbm_achieved_gbs"] = alg_b / sec / 1e9
             out["hbm_frac"] = out["hbm_achieved_gbs"] / peaks["hbm_gbs"]
         return out
+    if kind == "sentinels":        # reads a routed row's route + near-miss ids, writes the rest
+        alg = routed * w.c * 4
+        return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                    alg_per_launch=alg / launches)
     if kind == "compact":
         alg = (layer_calls - n_anchor) * w.rows + cnt["flagged_rows"] * 4
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
@@ -307,37 +332,32 @@ def run_ours(args) -> None:
     barrier()
     clocks = ClockSampler(local)
     launches0 = B.rr_kernel_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # L2: a step reads every layer's inputs once.  Where one step's inputs exceed L2 several
-    # times over nothing survives from step to step; smaller workloads get L2 flushed (a
-    # 256 MB buffer written) between steps, each step timed with its own pair of events.
+    # Every step is timed with its own pair of events on the launching stream; the reported
+    # step time is the median over the K steps (the paper's statistic), the mean is kept beside
+    # it.  L2: a step reads every layer's inputs once.  Where one step's inputs exceed L2
+    # several times over nothing survives from step to step; smaller workloads get L2 flushed
+    # (a 256 MB buffer written) before each step, outside its event pair.
     step_input_bytes = L * w.problems * (w.n_q + w.n_k) * w.d * esz
     flush_l2 = step_input_bytes < 2 * L2_BYTES
-    if flush_l2:
-        scratch = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-               for _ in range(args.steps)]
-        for a_ev, b_ev in evs:
+    scratch = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if flush_l2 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(args.steps)]
+    for a_ev, b_ev in evs:
+        if flush_l2:
             scratch.zero_()
-            a_ev.record(stream)
-            timed_step()
-            b_ev.record(stream)
-        barrier()
-        local_ms = sum(a_ev.elapsed_time(b_ev) for a_ev, b_ev in evs)
-        del scratch
-    else:
-        e0.record(stream)
-        for _ in range(args.steps):
-            timed_step()
-        e1.record(stream)
-        barrier()
-        local_ms = e0.elapsed_time(e1)
-    ms_total = max_over_ranks(local_ms, world, dev)
+        a_ev.record(stream)
+        timed_step()
+        b_ev.record(stream)
+    barrier()
+    step_ms = [a_ev.elapsed_time(b_ev) for a_ev, b_ev in evs]
+    del scratch
+    local_ms = statistics.median(step_ms)
+    mean_ms = max_over_ranks(sum(step_ms) / len(step_ms), world, dev)
+    ms_per_step = max_over_ranks(local_ms, world, dev)
     launches = B.rr_kernel_launch_count() - launches0
     if launches_per_replay is not None:
         launches = launches_per_replay * args.steps
     clock_info = clocks.stop()
-    ms_per_step = ms_total / args.steps
     value = aggregate_rows_per_s(w.rows, L, world, ms_per_step)
     if args.profile_only:            # short run for profiler captures: no extra passes
         if rank == 0:
@@ -438,14 +458,16 @@ def run_ours(args) -> None:
 
     step_e2e()
     barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
+    e2e_evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+    for a_ev, b_ev in e2e_evs:
+        a_ev.record(stream)
         step_e2e()
         stream.wait_stream(copy_stream)        # the step ends when its last routes are on the host
         stream.wait_stream(d2h_stream)
-    e1.record(stream)
+        b_ev.record(stream)
     barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    ms_e2e = max_over_ranks(statistics.median(a.elapsed_time(b) for a, b in e2e_evs), world, dev)
     h2d = L * w.problems * (w.n_q + w.n_k) * w.d * esz
     d2h = L * w.rows * w.k * 4
     e2e = {"value": aggregate_rows_per_s(w.rows, L, world, ms_e2e), "unit": UNIT,
@@ -453,17 +475,25 @@ def run_ours(args) -> None:
            "api": "rr_route_layers_host (copies overlapped on a second stream)"}
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) -----------------------------------------
-    cpu = None
+    cpu = cpu_timed = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, dt, summ, sample = _oracle_sample(w, 12, 9)
-        cpu = {"value": v, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
-               "sample": sample, "oracle_recall": summ.recall_all,
+        cpu = {"value": v, "unit": UNIT, "cores": _blas_threads(), "os_cpu_count": os.cpu_count(),
+               "kind": "oracle", "sample": sample, "oracle_recall": summ.recall_all,
                "oracle_flagged_fraction": summ.flagged_relay_fraction}
+        tp = min(w.problems, 4)
+        tv, tdt, tsample = _timed_sample(w, tp, w.layers)
+        cpu_timed = {"value": tv, "unit": UNIT, "cores": _blas_threads(),
+                     "os_cpu_count": os.cpu_count(), "kind": "oracle, vectorised fp32 timed mode "
+                     "(BLAS matmul + argpartition, gathered rescoring)", "sample": tsample}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_mean": mean_ms,
+            "ms_per_step_min": min(step_ms), "ms_per_step_max": max(step_ms),
+            "timing": "one CUDA-event pair per step; ms_per_step = median over steps, max "
+                      "over ranks", "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if w.dtype == W.DTYPE_BF16 else "f32", "data": "synthetic",
             "config": {"workload": w.name, "problems": w.problems, "n_q": w.n_q, "n_k": w.n_k,
@@ -476,7 +506,7 @@ def run_ours(args) -> None:
                        "graph": bool(args.graph),
                        "host_generation_s": round(t_gen, 1)},
             "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu,
+            "roofline": roofline, "cpu_baseline": cpu, "cpu_baseline_vectorised": cpu_timed,
             "layers": {"anchor_ms": anchor_ms, "relay_ms": relay_ms, "full_routing_ms": full_ms,
                        "anchor_rows_per_s": w.rows / anchor_ms * 1e3,
                        "relay_rows_per_s": w.rows / relay_ms * 1e3,
