@@ -292,7 +292,7 @@ template <int I0>
 __device__ __forceinline__ void filter_group(uint32_t& w, const uint32_t (&acc)[SLICE], float tau,
                                              uint32_t col0, uint32_t v, uint32_t w_end, bool inner) {
   const bool tight = __any_sync(0xFFFFFFFFu, w + 8u * ENTRY_PITCH > w_end);
-  (void)inner;
+  (void)inner;   // (a separate form for tiles that no row's mask cuts measured slower: more code)
   if (tight) filter_eight<I0, true, true>(w, acc, tau, col0, v, w_end);
   else filter_eight<I0, true, false>(w, acc, tau, col0, v, w_end);
 }
@@ -312,7 +312,7 @@ template <int D>
 __global__ void __launch_bounds__(NT, 1)
 route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
-                   uint32_t layer, int inplace, int hooks) {
+                   uint32_t layer, int inplace, int hooks, int cta_stride) {
   const bool force_hard = hooks & 1, force_timeout = hooks & 2;      // test hooks
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
@@ -322,6 +322,8 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   uint8_t* s_buf = (uint8_t*)ctl + CTL_BYTES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const CUtensorMap* const tmap_ptr = &tmap_k;   // address in parameter space (what TMA needs)
+  if (tid == 0) tma_prefetch_desc(tmap_ptr);     // first thing: the descriptor fetch takes a while
 #ifdef RR_PHASE_TIMING
   const long long cta_t0_ = clock64();
 #endif
@@ -381,9 +383,24 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     ctl->hard_n = 0;
     ctl->n_flagged = 0; ctl->n_cand = 0; ctl->v_flagged = 0ull;
     mbar_fence_init();
-    tma_prefetch_desc(&tmap_k);
   }
-  if (warp == 0) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+  if (warp == 1) tmem_alloc(&ctl->tmem_base, TMEM_COLS);   // (warp 0's first thread is busy with the barriers)
+  // The Kc loads depend on nothing but the number of key tiles (from the tile's last row: rows
+  // ascend inside a tile), and the ring's stages are all free: the producer fills the ring before
+  // the CTA's first barrier, while the Qc rows are on their way.
+  if (warp == 0) {
+    const int last_local = min(seg_hi - seg_lo, (tm + 1) * BM) - 1;
+    const int last_row = row_list ? row_list[seg_lo + last_local] - prob * p.n_q : last_local;
+    const int nt0 = (rr_valid_count(last_row, p.n_k, p.causal, p.causal_offset) + BN - 1) / BN;
+    if (lane == 0) {
+      const int pre = min(H_STAGES, 2 * nt0 * C::KHALVES);
+      for (int q = 0; q < pre; ++q) {
+        mbar_expect_tx(&ctl->full[q], C::B_HALF);
+        tma_load_3d(sB + q * C::B_HALF, tmap_ptr, (q % C::KHALVES) * 64, ((q / C::KHALVES) % nt0) * BN, prob, &ctl->full[q]);
+      }
+    }
+    __syncwarp();
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -391,19 +408,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   for (int t = BM - 1; t >= 0; --t) if (ctl->row[t] >= 0) { last = ctl->row[t]; break; }
   const int vmax = rr_valid_count(last, p.n_k, p.causal, p.causal_offset);
   const int n_tiles = (vmax + BN - 1) / BN;
-  const CUtensorMap* const tmap_ptr = &tmap_k;   // address in parameter space (what TMA needs)
-  // The Kc loads do not depend on the Qc tile: the ring's stages are filled (they are all free)
-  // and every Kc tile of the CTA is asked into L2 while the Qc rows are still on their way.
   const int pre_q = min(H_STAGES, 2 * n_tiles * C::KHALVES);
-  if (tid == 0) {
-    for (int q = 0; q < pre_q; ++q) {
-      mbar_expect_tx(&ctl->full[q], C::B_HALF);
-      tma_load_3d(sB + q * C::B_HALF, tmap_ptr, (q % C::KHALVES) * 64, ((q / C::KHALVES) % n_tiles) * BN, prob, &ctl->full[q]);
-    }
-    for (int t = 0; t < n_tiles; ++t)
-#pragma unroll
-      for (int h = 0; h < C::KHALVES; ++h) tma_prefetch_l2_3d(tmap_ptr, h * 64, t * BN, prob);
-  }
   if (q_loader) {
     const uint32_t taddr = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_COL;
     if constexpr (QW == 64) tmem_st_32x64(taddr, qv); else tmem_st_32x32(taddr, qv);
@@ -537,6 +542,27 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   if (warp == 0) {
     if (lane == 0) {
       produce(0, 2 * n_tiles, pre_q);
+    } else {
+      // every Kc tile of the CTA is asked into L2 (one prefetch per lane) ...
+      for (int q = lane - 1; q < n_tiles * C::KHALVES; q += 31)
+        tma_prefetch_l2_3d(tmap_ptr, (q % C::KHALVES) * 64, (q / C::KHALVES) * BN, prob);
+      // ... and so are the Qc rows of the CTA that will start about when this one ends (CTAs start in
+      // index order as SMs fall free, one CTA per SM) are asked into L2, so that its set-up waits
+      // for L2 instead of DRAM.  A hint only: nothing depends on it.
+      const int nb = (int)blockIdx.x + cta_stride;
+      if (nb < (int)gridDim.x) {
+        const int nprob = nb % p.P, ntm = tiles_m - 1 - nb / p.P;
+        int nlo = 0, nhi = p.n_q;
+        if (row_list) { nlo = p.problem_offsets[nprob]; nhi = p.problem_offsets[nprob + 1]; }
+        for (int i = lane - 1; i < BM; i += 31) {
+          const int local = ntm * BM + i;
+          if (local >= nhi - nlo) break;
+          const size_t grow = row_list ? (size_t)row_list[nlo + local] : (size_t)nprob * p.n_q + local;
+          const char* src = reinterpret_cast<const char*>(qc + grow * D);
+#pragma unroll
+          for (int b = 0; b < D * 2; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(src + b));
+        }
+      }
     }
     __syncwarp();
   } else if (!is_sel) {
@@ -778,11 +804,15 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     {
       const int my_d_max = __reduce_max_sync(FULL, my_d);
 #pragma unroll 1
-      for (int e = 0; e < my_d_max; ++e) {
-        if (e < my_d) {
-          const uint32_t id = lds32(my_base + (uint32_t)e * ENTRY_PITCH + 4u);
+      for (int e0 = 0; e0 < my_d_max; e0 += 4) {
+        uint32_t id[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) id[u] = lds32(my_base + (uint32_t)min(e0 + u, CAPJ - 1) * ENTRY_PITCH + 4u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = e0 + u;
           const int o = e < my_k ? off_k + e : p.k + off_n + (e - my_k);
-          sts32(stage_addr(o), id);
+          if (e < my_d) sts32(stage_addr(o), id[u]);
         }
       }
     }
@@ -881,9 +911,11 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 #ifdef RR_PHASE_TIMING
   if (tid == 0) { PH_CNT(14, clock64() - cta_t0_); PH_CNT(15, 1); }
 #endif
-  if (warp == 0) {
+  if (warp == 1) {                                         // the warp that allocated
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (warp == 0) {
     if (lane == 0 && ctl->abort_flag) atomicOr(p.status, RR_STATUS_TIMEOUT);
     if (lane == 0 && inplace) {      // what the compaction kernel and the work counters need
       p.tile_counts[prob * tiles_m + tm] = (int)ctl->n_flagged;
@@ -945,12 +977,15 @@ cudaError_t rr_launch_route_sweep(const RRParams& p, const void* qc, const void*
                                 227 * 1024);
   });
   if (e != cudaSuccess) return e;
+  int dev = 0, sms = 148;                     // CTAs resident at a time: one per SM
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const __nv_bfloat16* q = (const __nv_bfloat16*)qc;
   const size_t smem = smem_bytes(p.d);
   if (p.d == 128)
-    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks);
+    route_sweep_kernel<128><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks, sms);
   else
-    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks);
+    route_sweep_kernel<64><<<grid, NT, smem, st>>>(p, q, tmap, row_list, (uint32_t)layer, inplace, hooks, sms);
   rr_count_launch();
   return cudaPeekAtLastError();
 }
