@@ -251,6 +251,66 @@ int rr_compact_flags_noalloc(const uint8_t* dev_flags, int32_t n_problems, int32
                              int32_t* dev_rows_out, int32_t* dev_count_out,
                              int32_t* dev_problem_offsets_out, void* stream);
 
+/* ---- Route-width buckets (Section 4.4: "Ledgers are bucketed by route width so rows with
+ * compatible shapes share kernels"; Section 4.3: the ledger stores whichever route width the
+ * underlying policy requests) ------------------------------------------------------------------
+ * Problems (batch x head pairs) that ask for the same route width k form one bucket; a bucket is
+ * an ordinary ledger over its problems (same n_q, n_k, d, m, r, policies as cfg; cfg->k is
+ * ignored), and rr_bucket_route_layer runs every bucket's kernel set with one call per layer.
+ *
+ * Layout contract: Qc and Kc are laid out BUCKET-MAJOR -- the problems of bucket 0 first, then
+ * bucket 1, ... -- in the order rr_bucket_plan reports: buckets in ascending width, the problems
+ * of a bucket in ascending input index; order[s] = input index of the problem at slot s.  A
+ * bucket's inputs are then one contiguous [problems, n, d] block and nothing is gathered or
+ * copied.  Rows are numbered inside their bucket (position in the bucket * n_q + i); that id
+ * keys the sentinel sampler, so a bucket's results equal those of a stand-alone ledger (and of
+ * the method's definition) run on that bucket's problems alone.
+ * widths: host array [n_problems], 1 <= widths[p] <= n_k; n_problems = cfg->batch * cfg->heads.
+ * The set owns its ledgers' host handles, not the two device buffers (caller-owned, 256-byte
+ * aligned, at least the sizes rr_bucket_plan reports; bucket b uses the sub-ranges at
+ * rr_bucket_info.ledger_offset / scratch_offset). */
+typedef struct rr_bucket_set rr_bucket_set;
+typedef struct rr_bucket_info {
+  int32_t k;               /* route width of the bucket                                       */
+  int32_t problems;        /* how many problems it holds                                      */
+  int32_t first_slot;      /* bucket-major slot of its first problem                          */
+  size_t ledger_offset, scratch_offset, ledger_bytes, scratch_bytes;
+} rr_bucket_info;
+/* Host-only.  order_out [n_problems] (may be NULL), the number of buckets and the sizes of the
+ * two device buffers that hold all buckets. */
+int rr_bucket_plan(const rr_config* cfg, const int32_t* widths, int32_t n_problems,
+                   int32_t* order_out, int32_t* n_buckets_out, size_t* ledger_bytes,
+                   size_t* scratch_bytes);
+int rr_bucket_set_init(const rr_config* cfg, const int32_t* widths, int32_t n_problems,
+                       void* dev_ledger, size_t ledger_bytes, void* dev_scratch,
+                       size_t scratch_bytes, rr_bucket_set** out);
+int rr_bucket_set_destroy(rr_bucket_set* S);
+int rr_bucket_set_count(const rr_bucket_set* S);                 /* number of buckets (>= 1)    */
+int rr_bucket_set_info(const rr_bucket_set* S, int32_t b, rr_bucket_info* out);
+rr_ledger* rr_bucket_set_ledger(rr_bucket_set* S, int32_t b);    /* borrowed; for rr_ledger_views */
+int rr_bucket_set_reset(rr_bucket_set* S, void* stream);
+/* One layer for all buckets, enqueued on `stream` bucket after bucket.  qc / kc: device,
+ * bucket-major [P, n_q, d] / [P, n_k, d].  is_anchor != 0: anchor layer, else relay layer
+ * (RR_ERR_STATE before the first anchor). */
+int rr_bucket_route_layer(rr_bucket_set* S, const void* qc, const void* kc, int32_t layer,
+                          int32_t is_anchor, void* stream);
+/* OR of the buckets' status words; the first non-zero return of rr_ledger_status. Synchronous. */
+int rr_bucket_set_status(rr_bucket_set* S, void* stream, uint32_t* status_out);
+
+/* ---- A minimal consumer of token ranges (Eq. 3) ------------------------------------------------
+ * out[i] = softmax(q_i K_R^T * scale) V_R over the tokens R covered by row i's token ranges
+ * (views.token_ranges: [rows, slots, 2] = [start, end) per slot, (-1,-1) = empty; per route slot
+ * or coalesced).  One warp per row, FP32 arithmetic in ascending token order, so coalesced and
+ * per-slot ranges of the same route give bit-identical outputs.  A plain reference consumer, not
+ * a tuned attention backend (Section 4.3 leaves the backend unchanged); no token-level mask.
+ *   ranges  device int32 [rows, slots, 2]       q       device [rows, dh]
+ *   keys    device [rows / n_q, tokens, dh]      values  device, same shape as keys
+ *   dtype   RR_BF16 or RR_F32 (q, keys, values)  out     device float [rows, dh]
+ * A row without tokens gets zeros.  dh <= 256. */
+int rr_attend_token_ranges(const int32_t* ranges, int32_t rows, int32_t slots, int32_t n_q,
+                           const void* q, const void* keys, const void* values, int32_t tokens,
+                           int32_t dh, int32_t dtype, float scale, float* out, void* stream);
+
 /* Per-kernel device timing for benchmarks.  Between rr_profile_begin and rr_profile_end
  * every kernel the layer calls launch is bracketed by CUDA events on the caller's stream
  * (this adds event records to the stream; do not leave it on in production).

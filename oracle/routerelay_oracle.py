@@ -467,3 +467,25 @@ def token_ranges(routes: np.ndarray, chunk_tokens: int, coalesce: bool = False) 
             out[i, s, 1] = (j + 1) * chunk_tokens
             s += 1
     return out
+
+
+def routed_attention(q: np.ndarray, keys: np.ndarray, values: np.ndarray, routes: np.ndarray,
+                     chunk_tokens: int, scale: float) -> np.ndarray:
+    """Eq. 3: o_i = softmax(q_i K_R^T * scale) V_R, R = the tokens of the chunks in row i's route
+    (chunk j = tokens [j*T, (j+1)*T), clipped to the sequence).  One problem: q [n_q, dh],
+    keys / values [tokens, dh], routes [n_q, k] with -1 for empty slots.  float64; a row with an
+    empty route gets zeros."""
+    q = np.asarray(q, np.float64)
+    keys = np.asarray(keys, np.float64)
+    values = np.asarray(values, np.float64)
+    out = np.zeros((q.shape[0], values.shape[1]))
+    for i in range(q.shape[0]):
+        tok: List[int] = []
+        for j in sorted(set(int(c) for c in routes[i] if c >= 0)):
+            tok.extend(range(j * chunk_tokens, min((j + 1) * chunk_tokens, keys.shape[0])))
+        if not tok:
+            continue
+        logits = keys[tok] @ q[i] * scale
+        w = np.exp(logits - logits.max())
+        out[i] = (w / w.sum()) @ values[tok]
+    return out

@@ -49,6 +49,12 @@ class rr_views(C.Structure):
         "counters", "status")]
 
 
+class rr_bucket_info(C.Structure):
+    _fields_ = [("k", C.c_int32), ("problems", C.c_int32), ("first_slot", C.c_int32),
+                ("ledger_offset", C.c_size_t), ("scratch_offset", C.c_size_t),
+                ("ledger_bytes", C.c_size_t), ("scratch_bytes", C.c_size_t)]
+
+
 class RouteRelayError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -91,6 +97,24 @@ def lib() -> C.CDLL:
         L.rr_sampler_draw_u32.restype = C.c_uint32
         L.rr_compact_flags_noalloc.argtypes = [vp, i32, i32, vp, vp, vp, vp]
         L.rr_compact_flags_noalloc.restype = C.c_int
+        L.rr_bucket_plan.argtypes = [C.POINTER(rr_config), vp, i32, vp, C.POINTER(C.c_int32),
+                                     C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+        L.rr_bucket_set_init.argtypes = [C.POINTER(rr_config), vp, i32, vp, C.c_size_t, vp, C.c_size_t,
+                                         C.POINTER(vp)]
+        L.rr_bucket_set_destroy.argtypes = [vp]
+        L.rr_bucket_set_count.argtypes = [vp]
+        L.rr_bucket_set_info.argtypes = [vp, i32, C.POINTER(rr_bucket_info)]
+        L.rr_bucket_set_ledger.argtypes = [vp, i32]
+        L.rr_bucket_set_ledger.restype = vp
+        L.rr_bucket_set_reset.argtypes = [vp, vp]
+        L.rr_bucket_route_layer.argtypes = [vp, vp, vp, i32, i32, vp]
+        L.rr_bucket_set_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+        L.rr_attend_token_ranges.argtypes = [vp, i32, i32, i32, vp, vp, vp, i32, i32, i32, C.c_float,
+                                             vp, vp]
+        for name in ("rr_bucket_plan", "rr_bucket_set_init", "rr_bucket_set_destroy",
+                     "rr_bucket_set_count", "rr_bucket_set_info", "rr_bucket_set_reset",
+                     "rr_bucket_route_layer", "rr_bucket_set_status", "rr_attend_token_ranges"):
+            getattr(L, name).restype = C.c_int
         L.rr_profile_begin.argtypes = [vp]
         L.rr_profile_begin.restype = C.c_int
         L.rr_profile_end.argtypes = [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
@@ -214,6 +238,68 @@ def rr_compact_flags_noalloc(dev_flags: int, n_problems: int, n_q: int, dev_rows
     _check(lib().rr_compact_flags_noalloc(dev_flags, n_problems, n_q, dev_rows_out,
                                           dev_count_out, dev_problem_offsets_out, stream),
            "rr_compact_flags_noalloc")
+
+
+def rr_bucket_plan(cfg: rr_config, widths):
+    """(order, n_buckets, ledger_bytes, scratch_bytes) for the per-problem route widths."""
+    w = (C.c_int32 * len(widths))(*[int(x) for x in widths])
+    order = (C.c_int32 * len(widths))()
+    nb, a, b = C.c_int32(), C.c_size_t(), C.c_size_t()
+    _check(lib().rr_bucket_plan(C.byref(cfg), w, len(widths), order, C.byref(nb), C.byref(a),
+                                C.byref(b)), "rr_bucket_plan")
+    return list(order), nb.value, a.value, b.value
+
+
+def rr_bucket_set_init(cfg: rr_config, widths, dev_ledger: int, ledger_bytes: int,
+                       dev_scratch: int, scratch_bytes: int) -> int:
+    w = (C.c_int32 * len(widths))(*[int(x) for x in widths])
+    h = C.c_void_p()
+    _check(lib().rr_bucket_set_init(C.byref(cfg), w, len(widths), dev_ledger, ledger_bytes,
+                                    dev_scratch, scratch_bytes, C.byref(h)), "rr_bucket_set_init")
+    return h.value
+
+
+def rr_bucket_set_destroy(h: int) -> None:
+    _check(lib().rr_bucket_set_destroy(h), "rr_bucket_set_destroy")
+
+
+def rr_bucket_set_count(h: int) -> int:
+    n = lib().rr_bucket_set_count(h)
+    if n < 0:
+        _check(n, "rr_bucket_set_count")
+    return n
+
+
+def rr_bucket_set_info(h: int, b: int) -> rr_bucket_info:
+    info = rr_bucket_info()
+    _check(lib().rr_bucket_set_info(h, b, C.byref(info)), "rr_bucket_set_info")
+    return info
+
+
+def rr_bucket_set_ledger(h: int, b: int) -> int:
+    return lib().rr_bucket_set_ledger(h, b)
+
+
+def rr_bucket_set_reset(h: int, stream: int) -> None:
+    _check(lib().rr_bucket_set_reset(h, stream), "rr_bucket_set_reset")
+
+
+def rr_bucket_route_layer(h: int, qc: int, kc: int, layer: int, is_anchor: bool, stream: int) -> None:
+    _check(lib().rr_bucket_route_layer(h, qc, kc, layer, 1 if is_anchor else 0, stream),
+           "rr_bucket_route_layer")
+
+
+def rr_bucket_set_status(h: int, stream: int) -> int:
+    st = C.c_uint32()
+    _check(lib().rr_bucket_set_status(h, stream, C.byref(st)), "rr_bucket_set_status")
+    return st.value
+
+
+def rr_attend_token_ranges(ranges: int, rows: int, slots: int, n_q: int, q: int, keys: int,
+                           values: int, tokens: int, dh: int, dtype: int, scale: float, out: int,
+                           stream: int) -> None:
+    _check(lib().rr_attend_token_ranges(ranges, rows, slots, n_q, q, keys, values, tokens, dh,
+                                        dtype, scale, out, stream), "rr_attend_token_ranges")
 
 
 def rr_profile_begin(h: int) -> None:

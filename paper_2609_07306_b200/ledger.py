@@ -174,3 +174,90 @@ def device_tensor(x: np.ndarray, device="cuda:0") -> torch.Tensor:
     if x.dtype == np.uint16:
         return torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16)
     return torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(device)
+
+
+class _BucketLedger(RouteLedger):
+    """A bucket's ledger inside a BucketSet: same views and status calls as RouteLedger, but the
+    handle and the device buffers belong to the set."""
+
+    def __init__(self, handle: int, cfg: B.rr_config, ledger_buf, scratch_buf, device):
+        self.cfg, self.handle, self.device = cfg, handle, device
+        self.ledger_buf, self.scratch_buf = ledger_buf, scratch_buf
+        self.P = cfg.batch * cfg.heads
+        self.rows = self.P * cfg.n_q
+        self.sw = cfg.m + cfg.r + (cfg.global_sentinels & 1) + ((cfg.global_sentinels >> 1) & 1)
+        self.c = cfg.k + self.sw
+        self._views = B.rr_ledger_views(handle)
+
+    def close(self):
+        self.handle = None
+
+
+class BucketSet:
+    """Route-width buckets (Section 4.4): problems grouped by requested route width, one ledger
+    per bucket, one call per layer.  Inputs are bucket-major: use `order` to lay them out."""
+
+    def __init__(self, cfg: B.rr_config, widths, device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("BucketSet needs a CUDA device (there is no CPU path)")
+        self.cfg, self.device = cfg, torch.device(device)
+        self.order, n_buckets, lb, sb = B.rr_bucket_plan(cfg, widths)
+        with torch.cuda.device(self.device):
+            self.ledger_buf = torch.empty(lb + 256, dtype=torch.uint8, device=self.device)
+            self.scratch_buf = torch.empty(sb + 256, dtype=torch.uint8, device=self.device)
+            lo = (-self.ledger_buf.data_ptr()) % 256
+            so = (-self.scratch_buf.data_ptr()) % 256
+            self.handle = B.rr_bucket_set_init(cfg, widths, self.ledger_buf.data_ptr() + lo, lb,
+                                               self.scratch_buf.data_ptr() + so, sb)
+        assert B.rr_bucket_set_count(self.handle) == n_buckets
+        self.info = [B.rr_bucket_set_info(self.handle, b) for b in range(n_buckets)]
+        self.buckets = []
+        for b, inf in enumerate(self.info):
+            bc = B.rr_config()
+            C_fields = [f[0] for f in B.rr_config._fields_]
+            for f in C_fields:
+                setattr(bc, f, getattr(cfg, f))
+            bc.batch, bc.heads, bc.k = 1, inf.problems, inf.k
+            self.buckets.append(_BucketLedger(B.rr_bucket_set_ledger(self.handle, b), bc,
+                                              self.ledger_buf, self.scratch_buf, self.device))
+        self.reset()
+
+    def _stream(self) -> int:
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def reset(self):
+        B.rr_bucket_set_reset(self.handle, self._stream())
+
+    def route_layer(self, qc: torch.Tensor, kc: torch.Tensor, layer: int, is_anchor: bool):
+        B.rr_bucket_route_layer(self.handle, qc.data_ptr(), kc.data_ptr(), layer, is_anchor,
+                                self._stream())
+
+    def status(self) -> int:
+        return B.rr_bucket_set_status(self.handle, self._stream())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize(self.device)
+            B.rr_bucket_set_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def attend_token_ranges(ranges: torch.Tensor, n_q: int, q: torch.Tensor, keys: torch.Tensor,
+                        values: torch.Tensor, scale: float) -> torch.Tensor:
+    """Eq. 3 over the tokens the ranges cover (the library's reference consumer).
+    ranges [rows, slots, 2] int32; q [rows, dh]; keys / values [P, tokens, dh] (bf16 or fp32)."""
+    rows, slots = ranges.shape[0], ranges.shape[1]
+    dtype = {torch.bfloat16: B.RR_BF16, torch.float32: B.RR_F32}[q.dtype]
+    assert keys.dtype == q.dtype and values.dtype == q.dtype
+    assert ranges.is_contiguous() and q.is_contiguous() and keys.is_contiguous() and values.is_contiguous()
+    out = torch.empty((rows, q.shape[1]), dtype=torch.float32, device=q.device)
+    B.rr_attend_token_ranges(ranges.data_ptr(), rows, slots, n_q, q.data_ptr(), keys.data_ptr(),
+                             values.data_ptr(), keys.shape[1], q.shape[1], dtype, float(scale),
+                             out.data_ptr(), torch.cuda.current_stream(q.device).cuda_stream)
+    return out
