@@ -175,9 +175,22 @@ class ClockSampler:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels that
 # dominate a high_drift step, from the ncu captures summarised in profiles/
-# (route_fused_high_drift.md: 199.2 MB anchor / 204.3 MB refresh; rescore_dense_high_drift.md).
-NCU_TRAFFIC_BYTES = {"high_drift": {"route_fused": (4 * 199.3e6 + 28 * 200.6e6) / 32,
-                                    "rescore_dense": 244.2e6}}
+# (route_sweep_high_drift.md: 202.1 MB anchor / 216.8 MB refresh; rescore_dense_high_drift.md;
+# sentinels_high_drift.md), and the algorithmic bytes per launch of the same launches.  Other
+# workloads report the capture's traffic-to-algorithmic ratio times their own algorithmic bytes
+# and say so.
+NCU_TRAFFIC_BYTES = {"route_fused": ((4 * 202.1e6 + 28 * 216.8e6) / 32, (4 * 203.4e6 + 28 * 196.7e6) / 32),
+                     "rescore_dense": (241.3e6, 203.7e6),
+                     "sentinels": (66.6e6, 0.971 * 262144 * 64 * 4)}
+
+
+def _traffic(kind, workload_name, alg_bytes_per_launch, truncated):
+    if kind not in NCU_TRAFFIC_BYTES or alg_bytes_per_launch is None:
+        return None, None
+    measured, alg = NCU_TRAFFIC_BYTES[kind]
+    if workload_name == "high_drift" and not truncated:
+        return measured, "ncu capture (profiles/)"
+    return measured / alg * alg_bytes_per_launch, "scaled from the high_drift capture by algorithmic bytes"
 
 
 # ----------------------------------------------------------------------------- roofline
@@ -198,11 +211,11 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
     if kind == "topk_rows":        # reads score rows, writes ledger rows
         alg = cnt["full_pairs"] * 4 + routed * ledger_row
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                    alg_per_launch=alg / launches)
+                    alg_per_launch=alg / launches, alg_bytes_per_launch=alg / launches)
     if kind in ("rescore", "rescore_dense"):   # unique bytes: inputs + ledger ids + flags/alpha/beta
         alg = (layer_calls - n_anchor) * (in_bytes + w.rows * (w.c * 4 + 9))
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                    alg_per_launch=alg / launches)
+                    alg_per_launch=alg / launches, alg_bytes_per_launch=alg / launches)
     if kind == "score_simt":       # fp32 FMA: 2*d flop per score pair
         alg = 2.0 * w.d * cnt["full_pairs"]
         mhz = sm_mhz or 1965.0
@@ -219,18 +232,19 @@ def _kernel_roofline(kind, ms, launches, w, cnt, peaks, sm_mhz):
             alg_b = calls * in_bytes * (routed / (calls * w.rows)) + routed * ledger_row
             out["hbm_achieved_gbs"] = alg_b / sec / 1e9
             out["hbm_frac"] = out["hbm_achieved_gbs"] / peaks["hbm_gbs"]
+            out["alg_bytes_per_launch"] = alg_b / launches
         return out
     if kind == "sentinels":        # reads a routed row's route + near-miss ids, writes the rest
         alg = routed * w.c * 4
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                    alg_per_launch=alg / launches)
+                    alg_per_launch=alg / launches, alg_bytes_per_launch=alg / launches)
     if kind == "compact":
         alg = (layer_calls - n_anchor) * w.rows + cnt["flagged_rows"] * 4
         return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                    alg_per_launch=alg / launches)
+                    alg_per_launch=alg / launches, alg_bytes_per_launch=alg / launches)
     alg = layer_calls * w.rows * 9
     return dict(bound="hbm", achieved=alg / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                alg_per_launch=alg / launches)
+                alg_per_launch=alg / launches, alg_bytes_per_launch=alg / launches)
 
 
 # ----------------------------------------------------------------------------- multi-GPU plumbing
@@ -389,6 +403,11 @@ def run_ours(args) -> None:
         if "hbm_frac" in r:
             kernels[kind]["hbm_achieved_gbs"] = r["hbm_achieved_gbs"]
             kernels[kind]["hbm_frac"] = r["hbm_frac"]
+        kernels[kind]["alg_bytes_per_launch"] = r.get("alg_bytes_per_launch")
+        tr, src = _traffic(kind, w.name, r.get("alg_bytes_per_launch"), bool(args.layers))
+        if tr is not None:
+            kernels[kind]["traffic"] = tr
+            kernels[kind]["traffic_source"] = src
     top = next(iter(kernels))
     tk = kernels[top]
     roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
@@ -396,7 +415,8 @@ def run_ours(args) -> None:
                 "peak_source": (peaks["source"] + " (sustained bf16)" if tk["bound"] == "tensor"
                                 else peaks["source"]) if tk["bound"] != "alu" else
                 "148 SMs x 128 FMA/clk x 2 x sampled SM clock",
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(top) if not args.layers else None}
+                "traffic": tk.get("traffic"), "traffic_source": tk.get("traffic_source"),
+                "alg_bytes_per_launch": tk.get("alg_bytes_per_launch")}
     if "hbm_frac" in tk:
         roofline["hbm_achieved_gbs"] = tk["hbm_achieved_gbs"]
         roofline["hbm_frac"] = tk["hbm_frac"]
