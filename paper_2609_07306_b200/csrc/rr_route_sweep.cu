@@ -15,22 +15,25 @@
 //                scores of its row).
 // Sweep 1 (threshold before filtering): each thread keeps the running maximum of each of its
 // 32 column positions over all tiles -- 128 disjoint groups per row -- and sorts them with a
-// sorting network in registers.  With a = ceil(keep / 4), keep = k + max(m,1), the smallest of
-// the four threads' a-th largest group maxima has at least keep distinct scores of the row at
-// or above it, so it is a valid inclusive lower bound tau of the row's keep-th largest score
-// (about 1.4 keep scores pass).  A refresh row also has the bound the rescoring kernel derived
-// from its old candidates; the larger of the two is used.
+// sorting network in registers.  The keep-th largest of the row's 128 group maxima, keep =
+// k + max(m,1), has keep distinct scores of the row at or above it, so it is a valid inclusive
+// lower bound tau of the row's keep-th largest score, and the tightest the maxima give (about
+// 1.2 keep scores pass); one thread per row finds it by exchange over the four published sorted
+// lists (exchange_select).  A refresh row also has the bound the rescoring kernel derived from
+// its old candidates; the larger of the two is used.
 // Sweep 2 (the tile MMAs are simply issued again; Kc comes from L2): each thread appends its
 // scores >= tau to a private list of 32 {score, chunk id} entries in shared memory, sorts the
 // list (network on keys that carry 27 score bits and the list position, then an exact repair
-// of neighbours that agree in those bits) and writes it back in rank order.  One thread per row
-// then merges the row's four sorted lists from the top: the first k pops are the route, the
-// next m the near-miss sentinels, pop k+1 gives the margin.  Ties go to the smaller chunk id.
+// of neighbours that agree in those bits) and writes it back in rank order.  Two threads per row
+// then find, again by exchange over the row's four sorted lists, how many entries of each list
+// belong to the top k and to the top keep: the first give the route, the k-th score and the
+// margin, the rest the near-miss sentinels; every thread moves its own entries' ids to a staging
+// area and the ledger row goes out with 16-byte stores.  Ties go to the smaller chunk id.
 // The mandatory global and the random sentinels of the routed rows are built by a separate
 // one-thread-per-row kernel (rr_sentinels.cu) that runs at full occupancy: inside this kernel,
 // which holds one CTA per SM, their serial draws would sit on every CTA's critical path.
 // Rows the fast path cannot finish exactly (a list overflowed, three or more scores agreeing in
-// 27 bits inside one list) are handed to an exact slow path: one more sweep stores their
+// 27 bits inside one list, equal scores across a cut) are handed to an exact slow path: one more sweep stores their
 // complete score rows in shared memory, and a warp per row runs the radix select of the
 // two-pass path on them.  Every mbarrier wait is bounded.
 #include "rr_common.cuh"
