@@ -460,6 +460,41 @@ def run_ours(args) -> None:
     pairs = (c1["cand_pairs"] + c1["full_pairs"]) / c1["dense_pairs"]
     status = led.status()
 
+    # ---- the forced-anchor policy (Section 3.2) on the same inputs -----------------------------
+    # Relay calls that follow a tested relay with at least 90 % of the rows flagged route every
+    # row like an anchor (decided on the device; runs double up to 8 calls).  Not the headline:
+    # it shows what the schedule costs when the method itself notices that routes do not persist.
+    adaptive = None
+    if not args.inplace:
+        wa = w.replace(force_permille=args.force_permille, force_max_run=args.force_max_run)
+        aled = RouteLedger(config_from_workload(wa, two_pass=args.two_pass, gathered=args.gathered,
+                                                streaming=args.streaming), device=str(dev))
+
+        def astep():
+            for l in range(L):
+                (aled.route_anchor if w.is_anchor(l) else aled.route_relay)(dq[l], dk[l], l)
+
+        astep()
+        torch.cuda.synchronize()
+        forced0 = int(aled.force_state[4].item())
+        aev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(5)]
+        for a_ev, b_ev in aev:
+            a_ev.record(stream)
+            astep()
+            b_ev.record(stream)
+        torch.cuda.synchronize()
+        a_ms = max_over_ranks(statistics.median(a.elapsed_time(b) for a, b in aev), world, dev)
+        forced = (int(aled.force_state[4].item()) - forced0) / 5
+        n_anchor_l = sum(1 for l in range(L) if w.is_anchor(l))
+        relay_call_ms = (a_ms - n_anchor_l * anchor_ms) / max(1, L - n_anchor_l)
+        adaptive = {"force_permille": args.force_permille, "force_max_run": args.force_max_run,
+                    "ms_per_step": a_ms, "value": aggregate_rows_per_s(w.rows, L, world, a_ms),
+                    "forced_relay_calls_per_step": forced, "relay_calls_per_step": L - n_anchor_l,
+                    "mean_relay_call_ms": relay_call_ms,
+                    "relay_call_speedup_vs_full": full_ms / relay_call_ms}
+        aled.close()
+
     # ---- end to end: host buffers through rr_route_layers_host ------------------------------
     # (pinned host inputs copied in, every layer's routes copied back, copies overlapped with
     # the routing on a second stream -- all inside the library call)
@@ -532,6 +567,7 @@ def run_ours(args) -> None:
                        "relay_rows_per_s": w.rows / relay_ms * 1e3,
                        "full_routing_rows_per_s": w.rows / full_ms * 1e3,
                        "relay_speedup_vs_full": full_ms / relay_ms},
+            "adaptive_forced_anchors": adaptive,
             "quality": {"recall_vs_full_routing": hit / tot, "rerouted_row_fraction": rerouted,
                         "flagged_relay_row_fraction": flagged, "score_pair_fraction": pairs,
                         "status_word": status},
@@ -567,6 +603,10 @@ def main():
     ap.add_argument("--inplace", action="store_true",
                     help="relay layers: challenge test inside the routing kernel (one pass over "
                          "the score strip, no compacted second GEMM)")
+    ap.add_argument("--force-permille", type=int, default=900,
+                    help="forced-anchor policy of the extra 'adaptive_forced_anchors' pass: a tested "
+                         "relay that flags this many per mille of the rows forces the next ones")
+    ap.add_argument("--force-max-run", type=int, default=8)
     ap.add_argument("--gathered", action="store_true",
                     help="rescore candidates with the gathered FP32 kernel")
     args = ap.parse_args()

@@ -107,6 +107,18 @@ typedef struct rr_config {
   int32_t coalesce_ranges; /* with chunk_tokens > 0: runs of consecutive selected chunks become
                               one token range (the form a sparse-attention kernel consumes);
                               a row then holds its merged ranges first, (-1,-1) after them  */
+  int32_t force_permille;  /* forced anchors "before layers known to have low route
+                              persistence" (Section 3.2), decided on the device, no host round
+                              trip: >0 = a relay call whose challenge test flags at least
+                              ceil(rows * force_permille / 1000) rows makes the next relay
+                              calls route every row like an anchor (flags all 1, ages 0,
+                              sentinels redrawn, charged as anchor rows; the rescoring kernel
+                              exits at once).  While the flagged count stays that high the forced
+                              runs double -- 1, 2, 4, ... up to force_max_run calls -- with one
+                              tested call between two runs; a tested call below the threshold
+                              resets the run length; rr_route_anchor clears a pending run.
+                              0 = off.  Not available together with debug_outputs bit 5.      */
+  int32_t force_max_run;   /* longest forced run (values < 1 count as 1)                       */
 } rr_config;
 
 /* Device pointers into the caller's ledger/scratch buffers (valid until destroy). */
@@ -126,6 +138,9 @@ typedef struct rr_views {
   float*   cand_scores;     /* [rows, k+m+r+g] candidate scores of the last relay; NULL unless debug_outputs */
   uint64_t* counters;       /* [RR_NUM_COUNTERS] cumulative since reset, see below          */
   uint32_t* status;         /* [1]           RR_STATUS_* bits                               */
+  int32_t* force_state;     /* [8]           forced-anchor policy: words 0-3 = {pending forced calls,
+                                             run length} of the two call parities, 4 = forced calls
+                                             since reset, 5 = the last relay call was forced        */
 } rr_views;
 
 /* counters[] indices: work accounting in the sense of the paper's "rerouted rows" and
@@ -239,6 +254,9 @@ uint32_t rr_sampler_draw_u32(uint64_t seed, uint32_t g, uint32_t layer, uint32_t
  *
  * Limit: ceil(n_q / 128) * n_problems <= RR_NOALLOC_MAX_TILES (8.4 M rows when n_q is a
  * multiple of 128); larger inputs return RR_ERR_TOO_LARGE and nothing is enqueued.
+ * Cost: each 128-row tile's CTA re-sums the flagged counts of all earlier tiles (no waits between
+ * CTAs), n_tiles^2 / 2 four-byte reads from L2 in total: negligible at a few thousand tiles,
+ * milliseconds near the limit of 65536.
  * The call allocates nothing, on the host or the device, and only enqueues work on `stream`.
  * The first call on a device also looks up the array's device address (once per device,
  * with that device current); make that first call before starting any stream capture.

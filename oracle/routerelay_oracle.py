@@ -125,6 +125,10 @@ class OracleParams:
     gamma_boost: float = 0.0      # added to gamma while the row's recorded margin < margin_recover
     margin_recover: float = 0.0
     h_max: int = 0                # >0: a row last routed h_max or more layers ago is re-routed
+    # forced anchors before layers of low route persistence (Sec 3.2), decided from the flagged
+    # count of the last tested relay layer; 0 = off
+    force_permille: int = 0       # a tested relay that flags >= this many per mille of the rows ...
+    force_max_run: int = 1        # ... forces the next relay calls to route every row (see AnchorForcer)
 
     @property
     def n_global(self) -> int:
@@ -238,6 +242,7 @@ class LayerResult:
     full_routes: np.ndarray    # [rows, k] exact TopK of this layer (recall reference)
     scores: List[np.ndarray]   # per problem S (float64, masked)
     is_anchor: bool
+    forced: bool = False       # a relay call that the adaptive policy ran as an anchor
 
 
 def _problem_rows(p: OracleParams, slot: int) -> slice:
@@ -354,6 +359,45 @@ def relay_layer(prev: Ledger, q: np.ndarray, k: np.ndarray, p: OracleParams, lay
     return LayerResult(led, flags, alpha, beta, refresh_rows, cand_all, full, all_s, False)
 
 
+class AnchorForcer:
+    """Forced anchors "before layers known to have low route persistence" (Sec 3.2), with the
+    persistence read off the last tested relay layer.  State: `left` = relay calls still to be
+    run as forced anchors, `run` = length of the last forced run (back-off memory).
+
+    * a tested relay layer that flags F >= ceil(rows * force_permille / 1000) rows forces the next
+      `run` relay calls, run = min(max(1, 2 * previous run), force_max_run): while the flagged
+      count stays high the forced runs double, up to force_max_run, and one tested layer probes
+      between two runs; a tested layer below the threshold resets the back-off (run = 0);
+    * a forced relay call routes every row exactly like an anchor (flags all 1, ages 0, sentinels
+      redrawn at that layer) and decrements `left`;
+    * a scheduled anchor clears `left` and leaves `run`."""
+
+    def __init__(self, p: "OracleParams", rows: int):
+        self.on = p.force_permille > 0
+        self.threshold = (rows * p.force_permille + 999) // 1000
+        self.max_run = max(1, p.force_max_run)
+        self.left = 0
+        self.run = 0
+
+    def forced_now(self) -> bool:
+        return self.on and self.left > 0
+
+    def after_forced(self) -> None:
+        self.left -= 1
+
+    def after_anchor(self) -> None:
+        self.left = 0
+
+    def after_tested(self, flagged: int) -> None:
+        if not self.on:
+            return
+        if flagged >= self.threshold:
+            self.run = min(max(1, 2 * self.run), self.max_run)
+            self.left = self.run
+        else:
+            self.run = 0
+
+
 # --------------------------------------------------------------------------- metrics
 def recall_counts(routes: np.ndarray, full: np.ndarray):
     """(|route ∩ full| summed over rows, |full| summed over rows)."""
@@ -422,14 +466,23 @@ def run_layers(q_layers: np.ndarray, k_layers: np.ndarray, p: OracleParams,
     led: Optional[Ledger] = None
     kinds, flags_l, cc_l = [], [], []
     hit_all = tot_all = hit_rel = tot_rel = 0
+    forcer = AnchorForcer(p, P * p.n_q)
     for l in range(L):
         is_anchor = (l % anchor_every == 0)
         if is_anchor:
             res = anchor_layer(q_layers[l], k_layers[l], p, l, problem_ids)
             cc = None
+            forcer.after_anchor()
+        elif forcer.forced_now():                  # a relay call run as a forced anchor
+            res = anchor_layer(q_layers[l], k_layers[l], p, l, problem_ids)
+            res.forced = True
+            cc = None
+            is_anchor = True
+            forcer.after_forced()
         else:
             cc = valid_candidate_counts(led)
             res = relay_layer(led, q_layers[l], k_layers[l], p, l, problem_ids)
+            forcer.after_tested(int(res.flags.sum()))
         led = res.ledger
         h, t = recall_counts(led.routes, res.full_routes)
         hit_all += h

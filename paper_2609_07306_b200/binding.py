@@ -39,14 +39,15 @@ class rr_config(C.Structure):
                 ("chunk_tokens", C.c_int32), ("debug_outputs", C.c_int32),
                 ("global_sentinels", C.c_int32), ("min_reuse", C.c_int32), ("h_max", C.c_int32),
                 ("gamma_boost", C.c_float), ("margin_recover", C.c_float),
-                ("coalesce_ranges", C.c_int32)]
+                ("coalesce_ranges", C.c_int32), ("force_permille", C.c_int32),
+                ("force_max_run", C.c_int32)]
 
 
 class rr_views(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "routes", "sentinels", "ages", "kth_score", "margin", "flags", "alpha", "beta",
         "refresh_rows", "refresh_count", "problem_offsets", "token_ranges", "cand_scores",
-        "counters", "status")]
+        "counters", "status", "force_state")]
 
 
 class rr_bucket_info(C.Structure):

@@ -30,7 +30,7 @@ struct Layout {
   size_t routes, sentinels, ages, kth, margin, ledger_total;
   // scratch
   size_t flags, alpha, beta, tau, refresh_rows, refresh_count, problem_offsets, tile_counts,
-      token_ranges, cand_scores, counters, status, S, scratch_total;
+      token_ranges, cand_scores, counters, status, force_state, S, scratch_total;
   size_t export_total;
 };
 
@@ -50,6 +50,8 @@ int validate(const rr_config* c) {
   if (c->min_reuse < 0 || c->h_max < 0 || !(c->gamma_boost >= 0.f)) return RR_ERR_INVALID_ARG;
   if (c->margin_recover != c->margin_recover) return RR_ERR_INVALID_ARG;   // NaN
   if (c->coalesce_ranges != 0 && c->coalesce_ranges != 1) return RR_ERR_INVALID_ARG;
+  if (c->force_permille < 0 || c->force_permille > 1000) return RR_ERR_INVALID_ARG;
+  if (c->force_permille > 0 && (c->debug_outputs & 32)) return RR_ERR_UNSUPPORTED;
   if (c->k + c->m + c->r + (c->global_sentinels & 1) + ((c->global_sentinels >> 1) & 1) > RR_MAX_C)
     return RR_ERR_UNSUPPORTED;
   const long long rows = (long long)c->batch * c->heads * c->n_q;
@@ -112,6 +114,7 @@ Layout make_layout(const rr_config* c) {
   L.tile_counts = o;     o = align_up(o + tiles * 4);
   L.counters = o;        o = align_up(o + RR_NUM_COUNTERS * 8);
   L.status = o;          o = align_up(o + 4);
+  L.force_state = o;     o = align_up(o + 8 * 4);
   L.token_ranges = o;    o = align_up(o + (c->chunk_tokens > 0 ? rows * c->k * 8 : 0));
   L.cand_scores = o;     o = align_up(o + ((c->debug_outputs & 1) ? rows * cw * 4 : 0));
   // score rows are only materialised by the two-pass path
@@ -140,7 +143,10 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
                 cudaStream_t st) {
   if (!L || !qc || !kc || layer < 0) return RR_ERR_INVALID_ARG;
   if (!aligned16(qc) || !aligned16(kc)) return RR_ERR_INVALID_ARG;
-  const RRParams& p = L->p;
+  RRParams p = L->p;
+  p.force_in = p.force_stats + 2 * (L->call_index & 1u);
+  p.force_out = p.force_stats + 2 * ((L->call_index + 1u) & 1u);
+  ++L->call_index;
   // LAUNCH(kind, call): enqueue one kernel, bracketed by events while profiling
 #define LAUNCH(kind, call)                                                         \
   do {                                                                             \
@@ -270,6 +276,10 @@ int rr_ledger_init(const rr_config* cfg, void* dev_ledger, size_t ledger_bytes,
   p.tile_counts = (int32_t*)(sb + lay.tile_counts);
   p.counters = (unsigned long long*)(sb + lay.counters);
   p.status = (uint32_t*)(sb + lay.status);
+  p.force_stats = (int32_t*)(sb + lay.force_state);
+  p.force_in = p.force_out = p.force_stats;           // set per call (route_layer)
+  p.force_threshold = (int)(((long long)p.rows * cfg->force_permille + 999) / 1000);
+  p.force_max_run = cfg->force_max_run < 1 ? 1 : cfg->force_max_run;
   p.token_ranges = cfg->chunk_tokens > 0 ? (int32_t*)(sb + lay.token_ranges) : nullptr;
   p.cand_scores = (cfg->debug_outputs & 1) ? (float*)(sb + lay.cand_scores) : nullptr;
   p.S = (float*)(sb + lay.S);
@@ -285,6 +295,7 @@ int rr_ledger_reset(rr_ledger* L, void* stream) {
   if (!L) return RR_ERR_INVALID_ARG;
   RR_CUDA(rr_launch_reset(L->p, (cudaStream_t)stream));
   L->anchored = 0;
+  L->call_index = 0;
   return RR_OK;
 }
 
@@ -393,6 +404,7 @@ int rr_ledger_views(rr_ledger* L, rr_views* out) {
   out->refresh_count = p.refresh_count; out->problem_offsets = p.problem_offsets;
   out->token_ranges = p.token_ranges; out->cand_scores = p.cand_scores;
   out->counters = (uint64_t*)p.counters; out->status = p.status;
+  out->force_state = p.force_stats;
   return RR_OK;
 }
 

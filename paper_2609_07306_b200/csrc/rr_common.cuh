@@ -29,6 +29,11 @@ struct RRParams {
   int32_t* token_ranges; float* cand_scores;
   unsigned long long* counters; uint32_t* status;
   float* S;                                // [rows, n_k] score rows of the two-pass path
+  // forced anchors before layers of low route persistence (Section 3.2; 0 = off): a relay call
+  // reads {pending forced calls, run length} at force_in and writes the next call's pair at
+  // force_out (two slots, alternating per call, so that no CTA reads what another one writes)
+  int force_threshold, force_max_run;
+  int32_t* force_in; int32_t* force_out; int32_t* force_stats;
 };
 
 struct rr_ledger {
@@ -39,6 +44,7 @@ struct rr_ledger {
   size_t export_bytes;
   int device;
   int anchored;                            // host-side: has an anchor been enqueued since reset
+  unsigned call_index;                     // layer calls since reset (parity of the force_state slots)
   int timeout_shots;                       // test hook: forced time-outs still to be fired (bit 0
                                            // routing kernel, bit 1 strip rescoring kernel)
   bool sweep;                              // full routing runs in the two-sweep fused kernel

@@ -12,7 +12,8 @@ constexpr unsigned FULL = 0xFFFFFFFFu;
 // One CTA per row tile (RR_ROW_TILE rows of one problem).  The tile's base offset is the sum
 // of the flagged counts of all earlier tiles (written by the rescoring kernel); inside the
 // tile a ballot/popcount scan gives each flagged row its slot.  The list is therefore in
-// ascending global row id -- exactly numpy.nonzero(flags) -- with no atomics and no waits.
+// ascending global row id -- exactly numpy.nonzero(flags) -- with no atomics and no waits
+// (the price: n_tiles^2 / 2 count reads in total, nothing at the few thousand tiles of a layer).
 // The same pass advances the ages (flagged -> 0, stable -> +1) and, once per launch, the
 // per-layer counters: nothing later in the layer reads either.
 __global__ void __launch_bounds__(RR_ROW_TILE)
@@ -22,6 +23,35 @@ compact_kernel(RRParams p, unsigned long long dense_pairs) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_id = blockIdx.x;
   const int prob = tile_id / p.tiles_per_problem, tile = tile_id % p.tiles_per_problem;
+
+  // Forced anchor (Section 3.2, policy of rr_config.force_permille): the previous tested relay
+  // flagged so many rows that this call routes every row.  The tile does what the anchor's fill
+  // does for its rows; the rescoring kernel has exited without writing anything.
+  if (p.force_threshold > 0 && p.force_in[0] > 0) {
+    const int i = tile * RR_ROW_TILE + tid;
+    const int g = prob * p.n_q + i;
+    if (i < p.n_q) {
+      const float qnan = __int_as_float(0x7fc00000);
+      p.flags[g] = 1; p.refresh_rows[g] = g; p.ages[g] = 0;
+      p.alpha[g] = qnan; p.beta[g] = qnan; p.tau[g] = __int_as_float(0xff800000);
+    }
+    if (tid == 0) {
+      if (tile == 0) p.problem_offsets[prob] = prob * p.n_q;
+      if (tile_id == 0) {
+        p.counters[RR_CNT_LAYER_CALLS] += 1;
+        p.counters[RR_CNT_DENSE_PAIRS] += dense_pairs;
+        p.counters[RR_CNT_ANCHOR_ROWS] += (unsigned long long)p.rows;
+        p.counters[RR_CNT_FULL_PAIRS] += dense_pairs;
+      }
+      if (tile_id == p.n_tiles - 1) {
+        p.problem_offsets[p.P] = p.rows;
+        *p.refresh_count = p.rows;
+        p.force_out[0] = p.force_in[0] - 1; p.force_out[1] = p.force_in[1];
+        p.force_stats[4] += 1; p.force_stats[5] = 1;
+      }
+    }
+    return;
+  }
 
   int part = 0;
   for (int t = tid; t < tile_id; t += RR_ROW_TILE) part += p.tile_counts[t];
@@ -60,6 +90,10 @@ compact_kernel(RRParams p, unsigned long long dense_pairs) {
       for (int w = 0; w < RR_ROW_TILE / 32; ++w) total += s_part[w];
       p.problem_offsets[p.P] = total;
       *p.refresh_count = total;
+      if (p.force_threshold > 0) {    // this call was tested: decide about the next ones
+        const int run = total >= p.force_threshold ? min(max(1, 2 * p.force_in[1]), p.force_max_run) : 0;
+        p.force_out[0] = run; p.force_out[1] = run; p.force_stats[5] = 0;
+      }
     }
   }
 }
@@ -83,6 +117,9 @@ __global__ void anchor_fill_kernel(RRParams p, unsigned long long dense_pairs) {
     p.counters[RR_CNT_DENSE_PAIRS] += dense_pairs;
     p.counters[RR_CNT_ANCHOR_ROWS] += (unsigned long long)p.rows;
     p.counters[RR_CNT_FULL_PAIRS] += dense_pairs;
+    if (p.force_threshold > 0) {      // a scheduled anchor clears a pending forced run
+      p.force_out[0] = 0; p.force_out[1] = p.force_in[1]; p.force_stats[5] = 0;
+    }
   }
 }
 
@@ -177,6 +214,7 @@ __global__ void reset_kernel(RRParams p) {
   if (p.token_ranges)
     for (size_t e = tid; e < (size_t)p.rows * p.k * 2; e += stride) p.token_ranges[e] = -1;
   if (tid < RR_NUM_COUNTERS) p.counters[tid] = 0;
+  if (tid < 8) p.force_stats[tid] = 0;
   if (tid == 0) { *p.status = 0; *p.refresh_count = 0; }
 }
 

@@ -43,6 +43,7 @@ rescore_kernel(RRParams p, const T* __restrict__ qc, const T* __restrict__ kc) {
   constexpr int CPI = 32 / LPC;           // candidates per warp step
   __shared__ int s_flagged;
   __shared__ unsigned long long s_cand, s_full;
+  if (p.force_threshold > 0 && p.force_in[0] > 0) return;   // forced anchor: nothing is tested
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int prob = blockIdx.x / p.tiles_per_problem;
   const int tile = blockIdx.x % p.tiles_per_problem;

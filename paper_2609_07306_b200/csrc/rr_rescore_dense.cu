@@ -74,6 +74,7 @@ __global__ void __launch_bounds__(NT, 2)
 rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int words, int force_timeout) {
   using P = tcpipe::Pipe<D, BN, B_STAGES, ACC_STAGES, NCONS>;
+  if (p.force_threshold > 0 && p.force_in[0] > 0) return;   // forced anchor: nothing is tested
   extern __shared__ uint8_t smem_raw[];
   P pipe;
   pipe.carve(smem_raw);

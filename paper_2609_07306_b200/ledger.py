@@ -27,7 +27,8 @@ def config_from_workload(w: RouteWorkload, debug_outputs: bool = False,
                        global_sentinels=int(w.global_sentinels), min_reuse=int(w.min_reuse),
                        h_max=int(w.h_max), gamma_boost=float(w.gamma_boost),
                        margin_recover=float(w.margin_recover),
-                       coalesce_ranges=1 if w.coalesce_ranges else 0)
+                       coalesce_ranges=1 if w.coalesce_ranges else 0,
+                       force_permille=int(w.force_permille), force_max_run=int(w.force_max_run))
 
 
 class RouteLedger:
@@ -143,6 +144,9 @@ class RouteLedger:
     def token_ranges(self): return self._view("token_ranges", "i32", (self.rows, self.cfg.k, 2))
     @property
     def cand_scores(self): return self._view("cand_scores", "f32", (self.rows, self.c))
+    @property
+    def force_state(self): return self._view("force_state", "i32", (8,))
+
     @property
     def counters(self): return self._view("counters", "i64", (B.RR_NUM_COUNTERS,))
 

@@ -67,6 +67,8 @@ class RouteWorkload:
     gamma_boost: float = 0.0
     margin_recover: float = 0.0
     h_max: int = 0
+    force_permille: int = 0     # forced anchors after a relay that flags this many per mille of the rows
+    force_max_run: int = 1
 
     @property
     def problems(self) -> int:

@@ -36,7 +36,8 @@ def oracle_params(w: W.RouteWorkload) -> O.OracleParams:
                           causal=w.causal, causal_offset=w.causal_offset, seed=w.seed,
                           global_sentinels=w.global_sentinels, min_reuse=w.min_reuse,
                           gamma_boost=w.gamma_boost, margin_recover=w.margin_recover,
-                          h_max=w.h_max)
+                          h_max=w.h_max, force_permille=w.force_permille,
+                          force_max_run=w.force_max_run)
 
 
 def score_tol(qn: np.ndarray, kn_max: float, s_abs: np.ndarray) -> np.ndarray:

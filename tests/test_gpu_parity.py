@@ -447,3 +447,51 @@ def test_rectangular_shapes_of_the_paper(n_q, n_k):
         rep = parity.run_teacher_forced(w)
         _report(rep)
         parity.assert_clean(rep)
+
+
+@pytest.mark.parametrize("variant", ["default", "two_pass", "gathered"])
+def test_forced_anchors_after_low_persistence_follow_the_oracle(variant):
+    """Forced anchors before layers of low route persistence (Section 3.2), decided on the
+    device from the flagged count of the last tested relay: the sequence of tested / forced
+    calls, the work counters and the routes follow the oracle's run of the same policy."""
+    w = W.moderate().replace(force_permille=500, force_max_run=2, layers=12, anchor_every=6)
+    q, k = W.generate(w)
+    p = parity.oracle_params(w)
+    res, summ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),
+                             p, w.anchor_every)
+    want = [r.forced for r in res]
+    assert any(want) and not all(want[1:6])            # the policy fires and also probes
+    led = RouteLedger(config_from_workload(w, two_pass=(variant == "two_pass"),
+                                           gathered=(variant == "gathered")))
+    got = []
+    for l in range(w.layers):
+        fn = led.route_anchor if w.is_anchor(l) else led.route_relay
+        fn(device_tensor(q[l]), device_tensor(k[l]), l)
+        torch.cuda.synchronize()
+        st = led.force_state.cpu().numpy()
+        got.append(bool(st[5]))
+        if got[-1]:                                     # a forced call is an anchor in all but name
+            assert led.flags.all() and not led.ages.any()
+            assert int(led.refresh_count.item()) == w.rows
+            assert torch.equal(led.refresh_rows, torch.arange(w.rows, dtype=torch.int32, device="cuda"))
+        same = np.array([set(a) == set(b) for a, b in zip(led.routes.cpu().numpy(), res[l].ledger.routes)])
+        assert same.mean() > 0.99, (l, same.mean())
+    assert got == want
+    c = led.counters_dict()
+    assert c["anchor_rows"] == summ.counters["anchor_rows"]
+    assert c["relay_rows"] == summ.counters["relay_rows"]
+    assert abs(c["flagged_rows"] - summ.counters["flagged_rows"]) <= 0.01 * c["relay_rows"]
+    assert int(led.force_state[4].item()) == sum(want)
+    assert led.status() == 0
+    # reset clears the policy's state
+    led.reset()
+    torch.cuda.synchronize()
+    assert not led.force_state.any()
+    led.close()
+
+
+def test_forced_anchor_policy_is_refused_with_the_in_place_relay():
+    w = W.moderate().replace(force_permille=500)
+    with pytest.raises(B.RouteRelayError) as ei:
+        RouteLedger(config_from_workload(w, inplace=True))
+    assert ei.value.code == B.RR_ERR_UNSUPPORTED

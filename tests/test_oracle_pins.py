@@ -1,5 +1,6 @@
 """Pins for the CPU oracle: each test fixes the oracle to something other than itself
 (hand arithmetic, brute force, a lemma, a closed form, the paper's printed table)."""
+import dataclasses
 import math
 import os
 
@@ -525,3 +526,51 @@ def test_run_accounting_causal_candidate_pairs():
     # the per-row candidate count the run used equals the closed form slot by slot
     led = res[0].ledger
     assert np.array_equal(O.valid_candidate_counts(led), np.minimum(v, p.c))
+
+
+# ---- forced anchors before layers of low route persistence (Section 3.2) ---------------------
+def test_anchor_forcer_back_off_sequence_by_hand():
+    """Threshold 100 of 1000 rows, runs up to 4: T(high) F T(high) F F T(high) F F F F T(low) T(high) F."""
+    p = O.OracleParams(n_q=1000, n_k=8, k=1, m=1, r=0, force_permille=100, force_max_run=4)
+    f = O.AnchorForcer(p, 1000)
+    assert f.threshold == 100
+    trace = []
+    flagged = iter([100, 500, 999, 99, 100])          # what the tested layers see, in order
+    for _ in range(14):
+        if f.forced_now():
+            trace.append("F"); f.after_forced()
+        else:
+            trace.append("T"); f.after_tested(next(flagged, 0))
+    assert "".join(trace) == "TFTFFTFFFFTTFT"
+
+
+def test_anchor_forcer_threshold_rounds_up_and_scheduled_anchor_clears():
+    p = O.OracleParams(n_q=7, n_k=8, k=1, m=1, r=0, force_permille=500, force_max_run=2)
+    f = O.AnchorForcer(p, 7)
+    assert f.threshold == 4                            # ceil(3.5)
+    f.after_tested(3); assert not f.forced_now()
+    f.after_tested(4); assert f.forced_now() and f.left == 1
+    f.after_anchor(); assert not f.forced_now() and f.run == 1
+    f.after_tested(7); assert f.left == 2              # back-off memory survived the anchor
+    off = O.AnchorForcer(O.OracleParams(n_q=7, n_k=8, k=1, m=1, r=0), 7)
+    off.after_tested(7); assert not off.forced_now()
+
+
+def test_run_with_forced_anchors_routes_every_row_on_forced_layers():
+    """permille = 1 (any flagged row triggers), max run 1, strong drift: relay calls alternate
+    tested / forced; a forced layer equals full routing of that layer and resets every age."""
+    w = W.tiny().replace(rho=0.5, layers=6, anchor_every=6)
+    q, k = W.generate(w)
+    qf, kf = W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64)
+    p = O.OracleParams(n_q=w.n_q, n_k=w.n_k, k=w.k, m=w.m, r=w.r, seed=w.seed,
+                       force_permille=1, force_max_run=1)
+    res, summ = O.run_layers(qf, kf, p, w.anchor_every)
+    assert [r.forced for r in res] == [False, False, True, False, True, False]
+    assert [r.is_anchor for r in res] == [True, False, True, False, True, False]
+    for l in (2, 4):
+        assert np.array_equal(res[l].ledger.routes, res[l].full_routes)
+        assert not res[l].ledger.ages.any() and res[l].flags.all()
+    # forced layers are charged as anchors
+    assert summ.counters["anchor_rows"] == 3 * w.n_q and summ.counters["relay_rows"] == 3 * w.n_q
+    plain, _ = O.run_layers(qf, kf, dataclasses.replace(p, force_permille=0), w.anchor_every)
+    assert not any(r.forced for r in plain)
