@@ -15,10 +15,15 @@
 namespace {
 
 constexpr int NT = 64, WORDS = 32;             // rows per block; bitmap words per row (n_k <= 1024)
+constexpr int MAX_R = 32;                      // random sentinels staged per row (more: direct stores)
 
 __global__ void __launch_bounds__(NT)
 sentinel_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t layer) {
   __shared__ uint32_t s_bits[WORDS][NT];
+  // The row's random sentinels are collected here ([slot][thread]) and leave with 16-byte stores:
+  // the kernel is bound by the L1's sector accesses for its per-row (uncoalesced) traffic, and a
+  // 4-byte store per accepted draw costs one each.
+  __shared__ int32_t s_out[MAX_R][NT];
   const int tid = threadIdx.x;
   const int slot = blockIdx.x * NT + tid;
   const int count = row_list ? *p.refresh_count : p.rows;
@@ -65,6 +70,8 @@ sentinel_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t layer
   // ---- random sentinels ---------------------------------------------------------------------------
   int32_t* rnd = sent + p.m;
   int taken = 0;
+  const bool staged = p.r <= MAX_R && ((p.m | p.r | p.sw) & 3) == 0;
+  auto put = [&](int slot_, int id) { if (staged) s_out[slot_][tid] = id; else rnd[slot_] = id; };
   if (p.r > 0 && pool > 0) {
     if (pool > p.r) {
       const unsigned long long rk = rr_row_key(p.seed, (uint32_t)g);
@@ -80,15 +87,19 @@ sentinel_kernel(RRParams p, const int32_t* __restrict__ row_list, uint32_t layer
         for (int i = 0; i < 4; ++i) {
           const bool live = (t0 + i < limit) & (taken < p.r);
           const uint32_t w = s_bits[j4[i] >> 5][tid], bit = 1u << (j4[i] & 31);
-          if (live && !(w & bit)) { s_bits[j4[i] >> 5][tid] = w | bit; rnd[taken++] = j4[i]; }
+          if (live && !(w & bit)) { s_bits[j4[i] >> 5][tid] = w | bit; put(taken++, j4[i]); }
         }
       }
     }
     // whole pool (pool <= r) or the bounded-work fill: smallest free chunks first
     for (int j = 0; j < v && taken < p.r; ++j)
-      if (!((s_bits[j >> 5][tid] >> (j & 31)) & 1u)) rnd[taken++] = j;
+      if (!((s_bits[j >> 5][tid] >> (j & 31)) & 1u)) put(taken++, j);
   }
-  for (int e = taken; e < p.r; ++e) rnd[e] = -1;
+  for (int e = taken; e < p.r; ++e) put(e, -1);
+  if (staged)
+    for (int e = 0; e < p.r; e += 4)
+      *reinterpret_cast<int4*>(rnd + e) =
+          make_int4(s_out[e][tid], s_out[e + 1][tid], s_out[e + 2][tid], s_out[e + 3][tid]);
 }
 
 }  // namespace
