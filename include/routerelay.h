@@ -87,6 +87,9 @@ typedef struct rr_config {
                               the routing kernel on the scores of its first sweep (no separate
                               rescoring kernel, no second score GEMM over a compacted list);
                               the results are the same;
+                              bit 8: route with the two-sweep kernel whatever the grid size
+                              (by default grids of less than two waves of CTAs use the
+                              streaming kernel: fewer launches, shorter latency chain);
                               bits 6, 7 (tests): the first wait of the first CTA of the first
                               routing launch (bit 6) / strip rescoring launch (bit 7) of this
                               ledger counts as expired, once: that CTA gives up as after a real

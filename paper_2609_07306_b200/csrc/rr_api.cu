@@ -81,8 +81,16 @@ RRParams shape_params(const rr_config* cfg) {
   return p;
 }
 
+// The two-sweep kernel wins where the grid fills the GPU several times over (its per-score work
+// is smaller); on grids of less than two waves of CTAs a layer is a chain of kernel latencies,
+// and the streaming kernel -- one sweep, sentinels inside, one launch less -- is the shorter
+// chain (measured on the 32-problem chunk sweep: 5-10 % per step).  148 SMs, one CTA per SM.
 bool uses_sweep(const rr_config* cfg) {
-  return !(cfg->debug_outputs & (2 | 16)) && rr_route_sweep_supported(shape_params(cfg));
+  if (cfg->debug_outputs & (2 | 16)) return false;
+  const RRParams p = shape_params(cfg);
+  if (!rr_route_sweep_supported(p)) return false;
+  const bool forced = (cfg->debug_outputs & (32 | 256)) != 0;   // relay in place needs it; bit 8 asks for it
+  return forced || p.n_tiles >= 2 * 148 || !rr_route_fused_supported(p);
 }
 
 bool uses_fused(const rr_config* cfg) {

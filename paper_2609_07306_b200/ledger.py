@@ -14,7 +14,8 @@ _TORCH_DT = {"i32": torch.int32, "f32": torch.float32, "u8": torch.uint8, "i64":
 def config_from_workload(w: RouteWorkload, debug_outputs: bool = False,
                          two_pass: bool = False, gathered: bool = False,
                          force_slow_rows: bool = False, streaming: bool = False,
-                         inplace: bool = False, forced_timeouts: int = 0) -> B.rr_config:
+                         inplace: bool = False, forced_timeouts: int = 0,
+                         two_sweep: bool = False) -> B.rr_config:
     return B.rr_config(batch=w.batch, heads=w.heads, n_q=w.n_q, n_k=w.n_k, d=w.d, k=w.k, m=w.m,
                        r=w.r, dtype=B.RR_BF16 if w.dtype == DTYPE_BF16 else B.RR_F32,
                        causal=1 if w.causal else 0, causal_offset=int(w.causal_offset),
@@ -23,7 +24,7 @@ def config_from_workload(w: RouteWorkload, debug_outputs: bool = False,
                        debug_outputs=(1 if debug_outputs else 0) | (2 if two_pass else 0) |
                        (4 if gathered else 0) | (8 if force_slow_rows else 0) |
                        (16 if streaming else 0) | (32 if inplace else 0) |
-                       ((forced_timeouts & 3) << 6),
+                       ((forced_timeouts & 3) << 6) | (256 if two_sweep else 0),
                        global_sentinels=int(w.global_sentinels), min_reuse=int(w.min_reuse),
                        h_max=int(w.h_max), gamma_boost=float(w.gamma_boost),
                        margin_recover=float(w.margin_recover),

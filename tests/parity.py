@@ -80,7 +80,7 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
                        layers: Optional[int] = None, gen_threads: int = 8,
                        report: Optional[ParityReport] = None,
                        two_pass: bool = False, gathered: bool = False,
-                       force_slow_rows: bool = False, streaming: bool = False,
+                       force_slow_rows: bool = False, streaming: bool = False, two_sweep: bool = True,
                        inplace: bool = False) -> ParityReport:
     """Runs `layers` layers of workload w on the device over ALL problems and checks the
     listed problems (default all) against the oracle with teacher forcing."""
@@ -92,7 +92,8 @@ def run_teacher_forced(w: W.RouteWorkload, check_problems: Optional[Sequence[int
     q_all, k_all = W.generate(w, problems=all_problems, layers=L, threads=gen_threads)
     led = RouteLedger(config_from_workload(w, debug_outputs=True, two_pass=two_pass,
                                            gathered=gathered, force_slow_rows=force_slow_rows,
-                                           streaming=streaming, inplace=inplace))
+                                           streaming=streaming, inplace=inplace,
+                                           two_sweep=two_sweep))
     rows_sel = np.concatenate([np.arange(pr * w.n_q, (pr + 1) * w.n_q) for pr in check])
     sel_t = torch.from_numpy(rows_sel).cuda()
     v_sel = np.tile(p.valid_counts(), len(check))

@@ -62,12 +62,14 @@ def test_routing_kernel_variants(wl, variant):
     parity.assert_clean(rep)
 
 
-def test_degenerate_all_equal_scores_bf16():
-    """All-zero bf16 inputs through the fused routing kernel (every score ties, so every list of
-    the two-sweep kernel is one run of equal keys: all rows take its slow path): TopK must take
-    the smallest ids under the causal mask, margin 0."""
+@pytest.mark.parametrize("two_sweep", [True, False])
+def test_degenerate_all_equal_scores_bf16(two_sweep):
+    """All-zero bf16 inputs through the fused routing kernels (every score ties; in the two-sweep
+    kernel every list is one run of equal keys, so all rows take its slow path; a grid this small
+    uses the streaming kernel unless the two-sweep kernel is asked for): TopK must take the
+    smallest ids under the causal mask, margin 0."""
     w = W.moderate().replace(heads=2)
-    led = RouteLedger(config_from_workload(w))
+    led = RouteLedger(config_from_workload(w, two_sweep=two_sweep))
     z = torch.zeros(1, w.problems, w.n_q, w.d, device="cuda", dtype=torch.bfloat16)
     led.route_anchor(z, z, 0)
     torch.cuda.synchronize()

@@ -26,8 +26,9 @@ def _expect_timeout(led):
 def test_forced_timeout_is_reported_and_recoverable(which):
     w = W.moderate().replace(heads=2)
     q, k = W.generate(w, layers=2)
-    led = RouteLedger(config_from_workload(w, forced_timeouts=1 if which == "routing" else 2))
-    ref = RouteLedger(config_from_workload(w))
+    led = RouteLedger(config_from_workload(w, forced_timeouts=1 if which == "routing" else 2,
+                                          two_sweep=True))
+    ref = RouteLedger(config_from_workload(w, two_sweep=True))
     dq, dk = [device_tensor(x) for x in q], [device_tensor(x) for x in k]
     led.route_anchor(dq[0], dk[0], 0)
     ref.route_anchor(dq[0], dk[0], 0)
