@@ -196,48 +196,42 @@ __device__ __forceinline__ bool sort_list(uint32_t base, int n) {
 // move raises the sum of what is in, so the search ends, and it ends at the split that holds the
 // T largest scores: lo = the smallest score in (the T-th largest), hi = the largest score out.
 // Any split reached on the way already has T scores at or above its lo.
-// Two entries on either side of each cut are kept in registers, so a move is a register shuffle
-// and its refill load has a full step to arrive.  Warp-uniform: lanes that are done idle.
+// Every step re-reads the eight scores at the four cuts from shared memory (eight independent
+// loads) instead of carrying them in registers: the register form needs chains of selects to
+// address "the list that moves", and those chains, not the loads, were the step's latency.
+// Warp-uniform: lanes that are done idle.
 struct Exchange { int a0, a1, a2, a3; float lo, hi; };
-__device__ __forceinline__ float exch_score(uint32_t row_base, int j, int e, int nj) {
-  uint32_t bits;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(bits)
-               : "r"(row_base + (uint32_t)j * LIST_PITCH + (uint32_t)min(max(e, 0), CAPJ - 1) * ENTRY_PITCH)
-               : "memory");
-  return e < 0 ? __int_as_float(0x7f800000) : (e >= nj ? __int_as_float(0xff800000) : __uint_as_float(bits));
-}
 __device__ __forceinline__ Exchange exchange_select(uint32_t row_base, int n0, int n1, int n2, int n3,
                                                     int a0, int a1, int a2, int a3, bool on,
                                                     int max_steps) {
-  const float ninf = __int_as_float(0xff800000);
-#define RR_WIN(j) \
-  float p##j = exch_score(row_base, j, a##j - 2, n##j), l##j = exch_score(row_base, j, a##j - 1, n##j), \
-        x##j = exch_score(row_base, j, a##j, n##j), y##j = exch_score(row_base, j, a##j + 1, n##j);
-  RR_WIN(0) RR_WIN(1) RR_WIN(2) RR_WIN(3)
-#undef RR_WIN
-  float lo = fminf(fminf(l0, l1), fminf(l2, l3)), hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-  for (int it = 0; it < max_steps; ++it) {
-    const int jm = l0 == lo ? 0 : l1 == lo ? 1 : l2 == lo ? 2 : 3;
-    const float z0 = jm == 0 ? ninf : x0, z1 = jm == 1 ? ninf : x1;
-    const float z2 = jm == 2 ? ninf : x2, z3 = jm == 3 ? ninf : x3;
-    const float hz = fmaxf(fmaxf(z0, z1), fmaxf(z2, z3));
-    const int jx = z0 == hz ? 0 : z1 == hz ? 1 : z2 == hz ? 2 : 3;
-    const bool move = on && hz > lo;
-    if (!__any_sync(0xFFFFFFFFu, move)) break;
-    // refills: the entry two before the new cut of jm, the entry one behind the new cut of jx
-    const int am = jm == 0 ? a0 : jm == 1 ? a1 : jm == 2 ? a2 : a3;
-    const int ax = jx == 0 ? a0 : jx == 1 ? a1 : jx == 2 ? a2 : a3;
-    const int nx = jx == 0 ? n0 : jx == 1 ? n1 : jx == 2 ? n2 : n3;
-    const float rp = exch_score(row_base, jm, am - 3, CAPJ), ry = exch_score(row_base, jx, ax + 2, nx);
-    if (move) {
-#define RR_MOVE(j) \
-      if (jm == j) { y##j = x##j; x##j = l##j; l##j = p##j; p##j = rp; --a##j; } \
-      if (jx == j) { p##j = l##j; l##j = x##j; x##j = y##j; y##j = ry; ++a##j; }
-      RR_MOVE(0) RR_MOVE(1) RR_MOVE(2) RR_MOVE(3)
-#undef RR_MOVE
+  const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
+  float lo, hi;
+  for (int it = 0;; ++it) {
+    // last entry in (l) and first entry out (x) of every list; +inf / -inf where there is none
+#define RR_CUT(j)                                                                                   \
+    float l##j, x##j;                                                                               \
+    {                                                                                               \
+      const uint32_t base_ = row_base + (uint32_t)j * LIST_PITCH;                                   \
+      uint32_t lb_, xb_;                                                                            \
+      asm volatile("ld.shared.b32 %0, [%1];" : "=r"(lb_) : "r"(base_ + (uint32_t)max(a##j - 1, 0) * ENTRY_PITCH) : "memory"); \
+      asm volatile("ld.shared.b32 %0, [%1];" : "=r"(xb_) : "r"(base_ + (uint32_t)min(a##j, CAPJ - 1) * ENTRY_PITCH) : "memory"); \
+      l##j = a##j > 0 ? __uint_as_float(lb_) : pinf;                                                \
+      x##j = a##j < n##j ? __uint_as_float(xb_) : ninf;                                             \
     }
+    RR_CUT(0) RR_CUT(1) RR_CUT(2) RR_CUT(3)
+#undef RR_CUT
     lo = fminf(fminf(l0, l1), fminf(l2, l3));
     hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+    // the largest entry out cannot sit in the list of the smallest entry in (lists descend), so
+    // a strict gain always moves between two different lists
+    const bool move = on && hi > lo && it < max_steps;
+    if (!__any_sync(0xFFFFFFFFu, move)) break;
+    if (move) {
+      const int jm = l0 == lo ? 0 : l1 == lo ? 1 : l2 == lo ? 2 : 3;
+      const int jx = x0 == hi ? 0 : x1 == hi ? 1 : x2 == hi ? 2 : 3;
+      a0 += (jx == 0) - (jm == 0); a1 += (jx == 1) - (jm == 1);
+      a2 += (jx == 2) - (jm == 2); a3 += (jx == 3) - (jm == 3);
+    }
   }
   return Exchange{a0, a1, a2, a3, lo, hi};
 }
@@ -466,7 +460,7 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 #endif
       if (!mbar_wait_spin(&ctl->acc_empty[as], aph ^ 1, abort_flag)) break;
 #ifdef RR_PIPE_PROBE
-      PH_CNT(9, clock64() - ip0_); PH_CNT(14, 1);
+      PH_CNT(9, clock64() - ip0_); PH_CNT(13, 1);
 #endif
       bool ok = true;
 #pragma unroll
@@ -715,12 +709,12 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     bool slow = n_raw > CAPJ;                              // the list overflowed
     const int n = min(n_raw, CAPJ);
 
-    // ===== sort the list (network sized for the longest list of the warp) =========================
+    // ===== sort the list (network sized for the longest list of the warp; a third, smaller size
+    // cost more in code than it saved in compare-exchanges) ========================================
     {
       const int n_warp = __reduce_max_sync(FULL, n);
       bool run3;
-      if (n_warp <= 16) run3 = sort_list<16>(my_base, n);
-      else if (n_warp <= 24) run3 = sort_list<24>(my_base, n);
+      if (n_warp <= 24) run3 = sort_list<24>(my_base, n);
       else run3 = sort_list<32>(my_base, n);
       slow |= run3;
     }
