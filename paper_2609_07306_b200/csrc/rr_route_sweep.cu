@@ -537,13 +537,16 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
   auto acc_addr = [&](int gt) -> uint32_t { return acc_lane + (uint32_t)((gt % ACC_STAGES) * BN); };
 
   if (warp == 0) {
+    // Every Kc tile of the CTA beyond the ring is asked into L2, one prefetch per lane, BEFORE
+    // the first lane starts to produce: lanes of a warp whose first lane spins on a barrier may
+    // not get to run for a long time, and the hints are only worth something early.
+    for (int q = pre_q + lane; q < n_tiles * C::KHALVES; q += 32)
+      tma_prefetch_l2_3d(tmap_ptr, (q % C::KHALVES) * 64, (q / C::KHALVES) * BN, prob);
+    __syncwarp();
     if (lane == 0) {
       produce(0, 2 * n_tiles, pre_q);
     } else {
-      // every Kc tile of the CTA is asked into L2 (one prefetch per lane) ...
-      for (int q = lane - 1; q < n_tiles * C::KHALVES; q += 31)
-        tma_prefetch_l2_3d(tmap_ptr, (q % C::KHALVES) * 64, (q / C::KHALVES) * BN, prob);
-      // ... and so are the Qc rows of the CTA that will start about when this one ends (CTAs start in
+      // The Qc rows of the CTA that will start about when this one ends (CTAs start in
       // index order as SMs fall free, one CTA per SM) are asked into L2, so that its set-up waits
       // for L2 instead of DRAM.  A hint only: nothing depends on it.
       const int nb = (int)blockIdx.x + cta_stride;
@@ -898,7 +901,8 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
 
   // TMEM must not be freed while an MMA can still write to it: after a wait that gave up the
   // consumers no longer vouch for that, so each issuer waits (bounded) for its own MMAs
-  if (!is_sel && warp != 0 && lane == 0) {
+  // (when no wait gave up, every issued tile has been waited for by the consumers: nothing is pending)
+  if (!is_sel && warp != 0 && lane == 0 && ctl->abort_flag) {
     const int which = warp == 1 ? 0 : 1;
     umma_commit(&ctl->drain[which]);
     for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&ctl->drain[which], 0); ++it) __nanosleep(64);
