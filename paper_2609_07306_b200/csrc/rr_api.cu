@@ -198,7 +198,7 @@ int route_layer(rr_ledger* L, const void* qc, const void* kc, int layer, bool an
     if (L->dense_rescore) {
       const int shot = (L->timeout_shots >> 1) & 1;     // test hook: one forced time-out
       L->timeout_shots &= ~2;
-      LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, shot, st));
+      LAUNCH(RR_KIND_RESCORE_DENSE, rr_launch_rescore_dense(p, qc, kc, shot, /*prior=*/!L->sweep, st));
     }
     else LAUNCH(RR_KIND_RESCORE, rr_launch_rescore(p, qc, kc, st));
     LAUNCH(RR_KIND_COMPACT, rr_launch_compact(p, L->dense_pairs_per_layer, st));

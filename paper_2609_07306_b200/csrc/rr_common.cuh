@@ -134,7 +134,7 @@ cudaError_t rr_launch_rescore(const RRParams& p, const void* qc, const void* kc,
                               cudaStream_t st);
 bool rr_rescore_dense_supported(const RRParams& p);
 cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
-                                    int force_timeout, cudaStream_t st);
+                                    int force_timeout, bool prior, cudaStream_t st);
 // compact / anchor_fill also advance the ages and the cumulative counters of the layer
 cudaError_t rr_launch_compact(const RRParams& p, unsigned long long dense_pairs, cudaStream_t st);
 cudaError_t rr_launch_anchor_fill(const RRParams& p, unsigned long long dense_pairs,

@@ -69,7 +69,11 @@ __device__ unsigned long long g_rd_phase[8];
 // of a warp fall into 32 different banks whenever each thread touches a word of its own row).
 // Two planes encode the three candidate classes of a chunk:
 //   plane A | plane B :  route = 1|0,  near-miss = 0|1,  random sentinel = 1|1.
-template <int D>
+// PRIOR: also track the weakest near-miss candidate, so that tau = the floor of the k+m old
+// candidates' current scores can warm-start a refresh kernel that wants it (the streaming kernel;
+// the two-sweep kernel derives a tighter bound itself and the third masked pass is a tenth of
+// this kernel's time).
+template <int D, bool PRIOR>
 __global__ void __launch_bounds__(NT, 2)
 rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int words, int force_timeout) {
@@ -227,7 +231,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
           const float s0 = __uint_as_float(a0[q]);
           min_if(amin, s0, wr, 1u << q);
           max_if(bmax, s0, ws, 1u << q);
-          min_if(nmin, s0, wn, 1u << q);
+          if constexpr (PRIOR) min_if(nmin, s0, wn, 1u << q);
         }
       }
       if (p.debug) {                                         // tests: every candidate's score
@@ -270,7 +274,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
         p.flags[g] = flag ? 1 : 0;
         p.alpha[g] = amin;
         p.beta[g] = bmax;
-        p.tau[g] = p.m > 0 ? fminf(amin, nmin) : ninf;    // floor of the k+m old candidates
+        p.tau[g] = (PRIOR && p.m > 0) ? fminf(amin, nmin) : ninf;    // floor of the k+m old candidates
       }
       const int n_flag = __popc(__ballot_sync(FULL, flag));
       const int v_sum = __reduce_add_sync(FULL, flag ? v : 0);
@@ -314,7 +318,7 @@ bool rr_rescore_dense_supported(const RRParams& p) {
 }
 
 cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const void* kc,
-                                    int force_timeout, cudaStream_t st) {
+                                    int force_timeout, bool prior, cudaStream_t st) {
   int words;
   const size_t smem = smem_need(p, words);
   CUtensorMap tmap, tmap_q;
@@ -324,22 +328,24 @@ cudaError_t rr_launch_rescore_dense(const RRParams& p, const void* qc, const voi
   if (e != cudaSuccess) return e;
   static unsigned long long attr_done = 0;      // devices on which the attributes are set
   e = rr_once_per_device(attr_done, [] {
-    cudaError_t a = cudaFuncSetAttribute(rescore_dense_kernel<128>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (a != cudaSuccess) return a;
-    a = cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024);
-    if (a != cudaSuccess) return a;
-    cudaFuncSetAttribute(rescore_dense_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    cudaFuncSetAttribute(rescore_dense_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    const void* kernels[4] = {(const void*)rescore_dense_kernel<128, true>, (const void*)rescore_dense_kernel<128, false>,
+                              (const void*)rescore_dense_kernel<64, true>, (const void*)rescore_dense_kernel<64, false>};
+    for (const void* k : kernels) {
+      const cudaError_t a = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (a != cudaSuccess) return a;
+      cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    }
     return cudaSuccess;
   });
   if (e != cudaSuccess) return e;
   const int grid = p.n_tiles;
-  if (p.d == 128)
-    rescore_dense_kernel<128><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
-  else
-    rescore_dense_kernel<64><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
+  if (p.d == 128) {
+    if (prior) rescore_dense_kernel<128, true><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
+    else rescore_dense_kernel<128, false><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
+  } else {
+    if (prior) rescore_dense_kernel<64, true><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
+    else rescore_dense_kernel<64, false><<<grid, NT, smem, st>>>(p, tmap_q, tmap, words, force_timeout);
+  }
   rr_count_launch();
   return cudaPeekAtLastError();
 }

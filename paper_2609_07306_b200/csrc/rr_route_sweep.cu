@@ -19,8 +19,8 @@
 // k + max(m,1), has keep distinct scores of the row at or above it, so it is a valid inclusive
 // lower bound tau of the row's keep-th largest score, and the tightest the maxima give (about
 // 1.2 keep scores pass); one thread per row finds it by exchange over the four published sorted
-// lists (exchange_select).  A refresh row also has the bound the rescoring kernel derived from
-// its old candidates; the larger of the two is used.
+// lists (exchange_select).  (A bound from a refresh row's old candidates, as the streaming
+// kernel uses, bought nothing here and is not read.)
 // Sweep 2 (the tile MMAs are simply issued again; Kc comes from L2): each thread appends its
 // scores >= tau to a private list of 32 {score, chunk id} entries in shared memory, sorts the
 // list (network on keys that carry 27 score bits and the list position, then an exact repair
@@ -684,9 +684,6 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     PH_LAP(10);
     quarter_sync(quarter);                  // the published maxima have been read: lists are free
     tau = ctl->tau_row[r];
-    // rows of a refresh list also have the bound the rescoring kernel derived from the old
-    // candidates' current scores (bit-identical scores: no margin needed)
-    if (row_list && row >= 0) tau = fmaxf(tau, p.tau[g]);
     const bool routed = row >= 0 && (!inplace || ctl->live[r] != 0);   // this row is (re)routed here
     if (!routed) tau = pinf;                               // padding / reused rows pass nothing
     PH_LAP(1);
