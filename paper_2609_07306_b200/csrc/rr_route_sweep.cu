@@ -308,8 +308,12 @@ __device__ unsigned long long g_sweep_phase[32];
 template <int D>
 __global__ void __launch_bounds__(NT, 1)
 route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
-                   const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list,
+                   const __grid_constant__ CUtensorMap tmap_k, const int32_t* __restrict__ row_list_arg,
                    uint32_t layer, int inplace, int hooks, int cta_stride) {
+  // a relay call that the forced-anchor policy turned into full routing has the identity list:
+  // take the anchor's path (consecutive rows, no gathers through the list)
+  const int32_t* __restrict__ row_list =
+      (row_list_arg && p.force_threshold > 0 && p.force_in[0] > 0) ? nullptr : row_list_arg;
   const bool force_hard = hooks & 1, force_timeout = hooks & 2;      // test hooks
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
