@@ -312,8 +312,13 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
                    uint32_t layer, int inplace, int hooks, int cta_stride) {
   // a relay call that the forced-anchor policy turned into full routing has the identity list:
   // take the anchor's path (consecutive rows, no gathers through the list)
-  const int32_t* __restrict__ row_list =
-      (row_list_arg && p.force_threshold > 0 && p.force_in[0] > 0) ? nullptr : row_list_arg;
+  const bool forced_call = row_list_arg && p.force_threshold > 0 && p.force_in[0] > 0;
+  // A refresh list that holds nearly every row (high drift) is served the same way, with the
+  // rows that are not on it masked out: gathering 7/8 of the rows through the list costs more
+  // than sweeping the missing eighth for nothing (results per row are the same either way).
+  const bool dense_refresh = row_list_arg && !forced_call && !inplace &&
+                             (long long)(*p.refresh_count) * 8 >= (long long)p.rows * 7;
+  const int32_t* __restrict__ row_list = (forced_call || dense_refresh) ? nullptr : row_list_arg;
   const bool force_hard = hooks & 1, force_timeout = hooks & 2;      // test hooks
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
@@ -688,7 +693,8 @@ route_sweep_kernel(RRParams p, const __nv_bfloat16* __restrict__ qc,
     PH_LAP(10);
     quarter_sync(quarter);                  // the published maxima have been read: lists are free
     tau = ctl->tau_row[r];
-    const bool routed = row >= 0 && (!inplace || ctl->live[r] != 0);   // this row is (re)routed here
+    const bool routed = row >= 0 && (!inplace || ctl->live[r] != 0) &&      // this row is (re)routed here
+                        (!dense_refresh || p.flags[g] != 0);
     if (!routed) tau = pinf;                               // padding / reused rows pass nothing
     PH_LAP(1);
 
