@@ -175,12 +175,12 @@ class ClockSampler:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels that
 # dominate a high_drift step, from the ncu captures summarised in profiles/
-# (route_sweep_high_drift.md: 197.4 MB anchor / 217.2 MB refresh; rescore_dense_high_drift.md;
+# (route_sweep_high_drift.md: 199.1 MB anchor / 198.6 MB refresh; rescore_dense_high_drift.md;
 # sentinels_high_drift.md), and the algorithmic bytes per launch of the same launches.  Other
 # workloads report the capture's traffic-to-algorithmic ratio times their own algorithmic bytes
 # and say so.
-NCU_TRAFFIC_BYTES = {"route_fused": ((4 * 197.4e6 + 28 * 217.2e6) / 32, (4 * 203.4e6 + 28 * 196.7e6) / 32),
-                     "rescore_dense": (241.9e6, 203.7e6),
+NCU_TRAFFIC_BYTES = {"route_fused": ((4 * 199.1e6 + 28 * 198.6e6) / 32, (4 * 203.4e6 + 28 * 196.7e6) / 32),
+                     "rescore_dense": (242.8e6, 203.7e6),
                      "sentinels": (66.5e6, 0.971 * 262144 * 64 * 4)}
 
 
