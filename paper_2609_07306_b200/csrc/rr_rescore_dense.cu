@@ -101,10 +101,11 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
   // Each row has two consumer threads (warps 2-5: part 0, warps 6-9: part 1).  Part 0 owns
   // plane A of its row's bitmap (route and random / global sentinels), part 1 owns plane B
   // (all sentinels), so the two never write the same word and plain read-modify-writes do.
-  // A thread reads its ids 16 at a time (16-byte loads where the ledger row allows) and ORs
-  // them in groups of four: the four words are loaded together and ids that fall into the same
-  // word are chained in registers.  The first two batches are fetched before the pipeline
-  // set-up so that their memory round trip overlaps it.
+  // A thread reads its ids 16 at a time (16-byte loads where the ledger row allows) and sets
+  // their bits with shared-memory reductions (no read-modify-write round trips to wait for).
+  // The first two batches are fetched before the pipeline set-up so that their memory round
+  // trip overlaps it.  Without the prior-bound pass (PRIOR = false) the classes are just route
+  // (plane A) and sentinel (plane B): part 0 then skips the random / global slots.
   const int cquarter = warp & 3, cpart = (warp - 2) >> 2;
   const int crow_l = cquarter * 32 + lane;                       // row inside the tile
   const int crow = tm * tcpipe::BM + crow_l;
@@ -113,7 +114,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
   // part 0: range 0 = route [0, k), range 1 = sentinel slots [m, sw); part 1: range 0 = [0, sw)
   const int32_t* const ptr0 = cpart == 0 ? p.routes + cg * p.k : p.sentinels + cg * p.sw;
   const int32_t* const ptr1 = p.sentinels + cg * p.sw + p.m;
-  const int n0 = chas ? (cpart == 0 ? p.k : p.sw) : 0, n1 = chas && cpart == 0 ? p.sw - p.m : 0;
+  const int n0 = chas ? (cpart == 0 ? p.k : p.sw) : 0, n1 = chas && cpart == 0 && PRIOR ? p.sw - p.m : 0;
   auto load16 = [&](const int32_t* ptr, int s0, int n, int (&ids)[16]) {
     if (s0 + 16 <= n && (((uintptr_t)(ptr + s0)) & 15u) == 0) {
 #pragma unroll
@@ -162,30 +163,16 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
       // candidates are charged once: part 0 counts what it sets, part 1 only the near-miss slots
       auto or_ids = [&](const int (&ids)[16], int s0, int count_below) {
 #pragma unroll
-        for (int g0 = 0; g0 < 16; g0 += 4) {
-          uint32_t a[4], c[4], bit[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int id = ids[g0 + i];
-            bad |= id >= v;
-            const bool ok = id >= 0 && id < v;
-            a[i] = plane + (ok ? (uint32_t)(id >> 5) * 4u : 0u);
-            bit[i] = ok ? 1u << (id & 31) : 0u;
-            n_ok += ok && s0 + g0 + i < count_below;
-            c[i] = lds(a[i]);
-          }
-          uint32_t tot[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint32_t base = c[i];
-#pragma unroll
-            for (int h = 0; h < i; ++h) base = a[h] == a[i] ? tot[h] : base;
-            tot[i] = base | bit[i];
-            sts(a[i], tot[i]);
-          }
+        for (int i = 0; i < 16; ++i) {
+          const int id = ids[i];
+          bad |= id >= v;
+          const bool ok = id >= 0 && id < v;
+          n_ok += ok && s0 + i < count_below;
+          // a shared-memory reduction: the marks of a row do not wait for one another
+          if (ok) asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(plane + (uint32_t)(id >> 5) * 4u), "r"(1u << (id & 31)) : "memory");
         }
       };
-      const int cb0 = part == 0 ? 0x7fffffff : p.m;       // range 0: all / the near-miss slots
+      const int cb0 = (part == 0 || !PRIOR) ? 0x7fffffff : p.m;   // range 0: all / the near-miss slots
       or_ids(pre0, 0, cb0);
       or_ids(pre1, pre1_s0, pre1_is1 ? 0x7fffffff : cb0);
       const int n0_max = __reduce_max_sync(FULL, n0), n1_max = __reduce_max_sync(FULL, n1);
@@ -219,7 +206,7 @@ rescore_dense_kernel(RRParams p, const __grid_constant__ CUtensorMap tmap_q,
       const int wi = t * TPR + part;                       // this thread's word of either plane
       const bool in = alive && wi < words;
       const uint32_t wa = in ? lds(bA + wi * 4u) : 0u, wb = in ? lds(bB + wi * 4u) : 0u;
-      const uint32_t wr = wa & ~wb, wn = wb & ~wa, ws = wb;
+      const uint32_t wr = PRIOR ? wa & ~wb : wa, wn = wb & ~wa, ws = wb;
       const bool work = __any_sync(FULL, (wa | wb) != 0u);
       uint32_t a0[COLS];
       if (work) {

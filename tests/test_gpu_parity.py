@@ -309,8 +309,9 @@ def test_token_ranges(two_pass, coalesce):
     led.close()
 
 
+@pytest.mark.parametrize("two_sweep", [False, True], ids=["streaming", "two_sweep"])
 @pytest.mark.parametrize("wl", ["moderate", "sweep_1024_rho0.30_4heads"])
-def test_free_running_summary_matches_oracle(wl):
+def test_free_running_summary_matches_oracle(wl, two_sweep):
     """All layers without teacher forcing: recall / refreshed-row / score-pair fractions of
     the device run agree with the oracle's run up to the ambiguous rows.  Second case: the
     routing-scale sweep at 1024 chunks and the highest drift (4 of its 32 heads, 16 layers)."""
@@ -319,7 +320,7 @@ def test_free_running_summary_matches_oracle(wl):
     p = parity.oracle_params(w)
     res, summ = O.run_layers(W.as_float32(q).astype(np.float64), W.as_float32(k).astype(np.float64),
                              p, w.anchor_every)
-    led = RouteLedger(config_from_workload(w))
+    led = RouteLedger(config_from_workload(w, two_sweep=two_sweep))
     hit = tot = 0
     for l in range(w.layers):
         fn = led.route_anchor if w.is_anchor(l) else led.route_relay
