@@ -180,7 +180,7 @@ class ClockSampler:
 # workloads report the capture's traffic-to-algorithmic ratio times their own algorithmic bytes
 # and say so.
 NCU_TRAFFIC_BYTES = {"route_fused": ((4 * 199.1e6 + 28 * 198.6e6) / 32, (4 * 203.4e6 + 28 * 196.7e6) / 32),
-                     "rescore_dense": (242.8e6, 203.7e6),
+                     "rescore_dense": (241.3e6, 203.7e6),
                      "sentinels": (66.5e6, 0.971 * 262144 * 64 * 4)}
 
 
